@@ -22,9 +22,13 @@
  *     error nothing has been launched.
  *   - Every device-side wait is bounded.  If one gives up, the kernel records
  *     FA_ERR_DEVICE_TIMEOUT in a device status word, releases its tensor memory and exits;
- *     outputs are then undefined.  fa_last_device_status() reads that word; while it holds a
- *     timeout, every other unsatisfied wait of this library's kernels gives up as well (launches
- *     made before the word is read and cleared produce undefined outputs instead of waiting).
+ *     the outputs of THAT call are then undefined, and its other thread blocks stop waiting too.
+ *     fa_last_device_status() reads (and clears) the word.  Calls made after a timeout, read or
+ *     not, run normally: a recorded failure is tied to the launch that caused it.
+ *   - Host-side cost: the TMA tensor maps of a call (4 to 9, a microsecond or so each) are
+ *     encoded on every call; nothing is cached per pointer.  Per-device set-up (shared-memory
+ *     opt-in of the kernels, architecture check) is done once per device ordinal, so one process
+ *     may use the library on several GPUs (the device current at the call is the one used).
  */
 #ifndef FA_B200_H_
 #define FA_B200_H_
@@ -65,7 +69,7 @@ int fa_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
 size_t fa_bwd_workspace_bytes(int B, int H, int Hkv, int Sq, int Sk, int D);
 
 /*
- * Forward pass with different query/key and value head dimensions (Section 4.1 benchmarks head
+ * Forward pass with different query/key and value head dimensions (Section 5 benchmarks head
  * dimensions (192, 128) beside 64 and 128).  q: [B, Sq, H, Dqk], k: [B, Sk, Hkv, Dqk],
  * v: [B, Sk, Hkv, Dv], o: [B, Sq, H, Dv], lse: [B, H, Sq]; everything else as fa_fwd, including the
  * definition of scale (the caller passes it; 1/sqrt(Dqk) is customary) and the status codes.
@@ -157,7 +161,7 @@ int fa_bwd_deterministic(const void* q, const void* k, const void* v, const void
                          void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * FP16 variants (the paper's kernels take FP16 or BF16 inputs, Section 4.1): q, k, v, o, d_o, dq,
+ * FP16 variants (the paper's kernels take FP16 or BF16 inputs, Section 5): q, k, v, o, d_o, dq,
  * dk, dv hold IEEE half-precision elements instead of bfloat16; everything else - layouts, lse,
  * workspace, stream, status codes - is as in fa_fwd / fa_bwd.  Both support D in {64, 128} (a
  * process running with FA_BWD_IMPL=pair gets FA_ERR_UNSUPPORTED from fa_bwd_f16).  Probabilities

@@ -276,11 +276,6 @@ def fa_exp2_emulated(x, stream=None):
 BWD_LAUNCHES = 3  # kernels fa_bwd enqueues: preprocess, main, dQ conversion
 
 
-def has_backward():
-    """True once fa_bwd is implemented in the loaded library (it answers UNSUPPORTED until then)."""
-    return True
-
-
 BWD_NOALLOC_MAX_BYTES = 40 * 1024 * 1024
 
 

@@ -4,6 +4,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "exp2_emu.cuh"
@@ -16,6 +17,11 @@ int env_int(const char* name, int deflt) {
   const char* v = getenv(name);
   if (!v || !*v) return deflt;
   return atoi(v);
+}
+
+unsigned next_launch_epoch() {
+  static std::atomic<unsigned> counter{0};
+  return counter.fetch_add(1, std::memory_order_relaxed) + 1;  // never 0 in the first 2^32 - 1 calls
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -62,21 +68,26 @@ static int check_shape(int B, int H, int Hkv, int Sq, int Sk, int D, float scale
   return FA_OK;
 }
 
-// The kernels are built for sm_100a only; anything else (or no device at all) is refused.
+// The kernels are built for sm_100a only; anything else (or no device at all) is refused.  The
+// answer belongs to the current device and is cached per device ordinal (1 = supported, 2 = not).
 static int check_device() {
-  static int cached = -1;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    int dev = 0;
-    cudaDeviceProp prop;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+  static PerDeviceFlag verdict;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    cudaGetLastError();
+    return FA_ERR_CUDA;
+  }
+  int v = verdict.get(dev);
+  if (v == 0) {
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
       cudaGetLastError();
-      cached = FA_ERR_CUDA;
-      return;
+      return FA_ERR_CUDA;
     }
-    cached = (prop.major == 10) ? FA_OK : FA_ERR_UNSUPPORTED;
-  });
-  return cached;
+    v = major == 10 ? 1 : 2;
+    verdict.set(dev, v);
+  }
+  return v == 1 ? FA_OK : FA_ERR_UNSUPPORTED;
 }
 
 __global__ void exp2_emulated_kernel(const float* __restrict__ x, float* __restrict__ y, size_t n) {
@@ -86,16 +97,17 @@ __global__ void exp2_emulated_kernel(const float* __restrict__ x, float* __restr
 
 // One warp waits on a barrier that nobody arrives on: the bounded wait has to give up, record the
 // timeout in the device status word and let the kernel end normally.
-__global__ void unsatisfied_wait_kernel() {
+__global__ void unsatisfied_wait_kernel(unsigned epoch) {
   __shared__ alignas(8) uint64_t bar;
-  __shared__ int abort_flag;
+  __shared__ WaitCtl ctl;
   if (threadIdx.x == 0) {
-    abort_flag = 0;
+    ctl.abort_flag = 0;
+    ctl.launch_epoch = (int)epoch;
     mbar_init(&bar, 1);
     fence_barrier_init();
   }
   __syncthreads();
-  mbar_wait(&bar, 0, &abort_flag, __LINE__);
+  mbar_wait(&bar, 0, &ctl.abort_flag, __LINE__);
 }
 
 }  // namespace fa
@@ -267,13 +279,16 @@ const char* fa_status_string(int status) {
 
 int fa_last_device_status(void* stream) {
   if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return FA_ERR_CUDA;
-  int h = 0;
-  if (cudaMemcpyFromSymbol(&h, g_device_status, sizeof(int)) != cudaSuccess) return FA_ERR_CUDA;
+  unsigned long long word = 0;
+  if (cudaMemcpyFromSymbol(&word, g_device_status, sizeof(word)) != cudaSuccess) return FA_ERR_CUDA;
+  const unsigned h = (unsigned)word;
   if (h != 0) {
-    int zero = 0;
-    cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int));
+    const unsigned long long zero = 0;
+    cudaMemcpyToSymbol(g_device_status, &zero, sizeof(zero));
     // FA_LOG=1: say which wait gave up (source line of the kernel file), for bug reports
-    if (env_int("FA_LOG", 0)) fprintf(stderr, "fa: device-side wait expired (code %d, site %d)\n", h & 0xff, h >> 8);
+    if (env_int("FA_LOG", 0))
+      fprintf(stderr, "fa: device-side wait expired (code %u, site %u, launch %u)\n", h & 0xffu, h >> 8,
+              (unsigned)(word >> 32));
   }
   return h == 0 ? FA_OK : FA_ERR_DEVICE_TIMEOUT;
 }
@@ -291,7 +306,7 @@ int fa_exp2_emulated(const float* x, float* y, size_t n, void* stream) {
 int fa_selftest_unsatisfied_wait(void* stream) {
   int st = check_device();
   if (st != FA_OK) return st;
-  unsatisfied_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>();
+  unsatisfied_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(next_launch_epoch());
   return cudaGetLastError() == cudaSuccess ? FA_OK : FA_ERR_CUDA;
 }
 

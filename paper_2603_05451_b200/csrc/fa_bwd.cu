@@ -55,26 +55,21 @@ static BwdWorkspace bwd_layout(const Shape& s) {
 
 size_t bwd_workspace_bytes(const Shape& s) { return bwd_layout(s).total; }
 
-template <typename Kernel>
-static int set_smem(Kernel kernel, int bytes, bool* done) {
-  if (*done) return FA_OK;
-  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess)
-    return FA_ERR_CUDA;
-  *done = true;
-  return FA_OK;
-}
+// Shared-memory opt-in of the fused kernel (dense and packed launches share it), per device.
+static PerDeviceFlag g_attr_fused_bf16, g_attr_fused_f16;
 
 // The two split kernels: dK/dV per key tile, then dQ per query tile.
-template <int D, bool kF16>
+template <int D, bool kF16, typename Preprocess>
 static int bwd_split_launch(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
                             const CUtensorMap& tdq, const CUtensorMap& tdk, const CUtensorMap& tdv, const BwdParams& p,
-                            int n_kv_tiles, int n_q_tiles, cudaStream_t stream) {
+                            int n_kv_tiles, int n_q_tiles, Preprocess preprocess, cudaStream_t stream) {
   const long long n_kv_ctas = (long long)n_kv_tiles * p.Hkv * p.B;
   const long long n_q_ctas = (long long)n_q_tiles * p.H * p.B;
-  static bool attr_a = false, attr_b = false;
+  static PerDeviceFlag attr_a, attr_b;
   int st;
-  if ((st = set_smem(bwd_dkdv_kernel<D, kF16>, (int)sizeof(BwdDkdvSmem<D>), &attr_a)) != FA_OK) return st;
-  if ((st = set_smem(bwd_dq_kernel<D, kF16>, (int)sizeof(BwdDqSmem<D>), &attr_b)) != FA_OK) return st;
+  if ((st = set_smem_once(bwd_dkdv_kernel<D, kF16>, (int)sizeof(BwdDkdvSmem<D>), attr_a)) != FA_OK) return st;
+  if ((st = set_smem_once(bwd_dq_kernel<D, kF16>, (int)sizeof(BwdDqSmem<D>), attr_b)) != FA_OK) return st;
+  if ((st = preprocess()) != FA_OK) return st;
   bwd_dkdv_kernel<D, kF16><<<(unsigned)n_kv_ctas, 512, sizeof(BwdDkdvSmem<D>), stream>>>(tq, tk, tv, tdo, tdk, tdv, p,
                                                                                           n_kv_tiles);
   if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
@@ -104,19 +99,6 @@ static int bwd_launch_d(const void* q, const void* k, const void* v, const void*
   if ((st = encode_bshd_map(&tdk, dk, s.B, s.Sk, s.Hkv, D, 64, 128, bf16, 2, sw)) != FA_OK) return st;
   if ((st = encode_bshd_map(&tdv, dv, s.B, s.Sk, s.Hkv, D, 64, 128, bf16, 2, sw)) != FA_OK) return st;
 
-  // 1. preprocess: Delta, LSE in base 2 (and a zeroed dQ accumulator for the fused path)
-  {
-    constexpr int kRowsPerBlock = 256 / (D / 8);
-    const long long rows = (long long)s.B * s.H * w.sq_pad;
-    const long long blocks = (rows + kRowsPerBlock - 1) / kRowsPerBlock;
-    if (blocks > 0x7fffffffll) return FA_ERR_UNSUPPORTED;
-    auto pre = s.f16 ? bwd_preprocess_kernel<D, true> : bwd_preprocess_kernel<D, false>;
-    pre<<<(unsigned)blocks, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(o),
-                                              static_cast<const __nv_bfloat16*>(d_o), lse, delta, lse2, dq_acc, s.B,
-                                              s.H, s.Sq, w.sq_pad);
-    if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
-  }
-
   BwdParams p;
   p.dq_acc = dq_acc;
   p.lse2 = lse2;
@@ -125,11 +107,27 @@ static int bwd_launch_d(const void* q, const void* k, const void* v, const void*
   p.scale = s.scale;
   p.scale_log2 = s.scale * kLog2e;
   p.causal = s.causal;
+  p.epoch = next_launch_epoch();
   const int n_kv_tiles = (s.Sk + 127) / 128;
   const int n_q_tiles = (s.Sq + 127) / 128;
   const long long n_kv_ctas = (long long)n_kv_tiles * s.Hkv * s.B;
   const long long n_q_ctas = (long long)n_q_tiles * s.H * s.B;
-  if (n_kv_ctas > 0x7fffffffll || n_q_ctas > 0x7fffffffll) return FA_ERR_UNSUPPORTED;
+  // Every size check comes before the first launch: on an error nothing has been launched.
+  constexpr int kRowsPerBlock = 256 / (D / 8);
+  const long long pre_blocks = ((long long)s.B * s.H * w.sq_pad + kRowsPerBlock - 1) / kRowsPerBlock;
+  const size_t n8 = (size_t)s.B * s.Sq * s.H * D / 8;
+  const size_t conv_blocks = (n8 + 255) / 256;
+  if (n_kv_ctas > 0x3fffffffll || n_q_ctas > 0x7fffffffll || pre_blocks > 0x7fffffffll || conv_blocks > 0x7fffffffull)
+    return FA_ERR_UNSUPPORTED;
+
+  // 1. preprocess: Delta, LSE in base 2 (and a zeroed dQ accumulator for the fused path)
+  auto preprocess = [&]() {
+    auto pre = s.f16 ? bwd_preprocess_kernel<D, true> : bwd_preprocess_kernel<D, false>;
+    pre<<<(unsigned)pre_blocks, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(o),
+                                                  static_cast<const __nv_bfloat16*>(d_o), lse, delta, lse2, dq_acc, s.B,
+                                                  s.H, s.Sq, w.sq_pad);
+    return cudaGetLastError() == cudaSuccess ? FA_OK : FA_ERR_CUDA;
+  };
 
   if constexpr (D == 128) {
     if (fused) {
@@ -138,39 +136,36 @@ static int bwd_launch_d(const void* q, const void* k, const void* v, const void*
         CUtensorMap tq64, tdo64;
         if ((st = encode_bshd_map(&tq64, q, s.B, s.Sq, s.H, D, 64, 64, bf16, 2, sw)) != FA_OK) return st;
         if ((st = encode_bshd_map(&tdo64, d_o, s.B, s.Sq, s.H, D, 64, 64, bf16, 2, sw)) != FA_OK) return st;
-        static bool attr_p = false;
-        if ((st = set_smem(bwd_pair_kernel, (int)sizeof(BwdPairSmem), &attr_p)) != FA_OK) return st;
+        static PerDeviceFlag attr_p;
+        if ((st = set_smem_once(bwd_pair_kernel, (int)sizeof(BwdPairSmem), attr_p)) != FA_OK) return st;
         const int n_kv_pairs = (n_kv_tiles + 1) / 2;
-        const long long n_pair_ctas = 2ll * n_kv_pairs * s.Hkv * s.B;
-        if (n_pair_ctas > 0x7fffffffll) return FA_ERR_UNSUPPORTED;
+        const long long n_pair_ctas = 2ll * n_kv_pairs * s.Hkv * s.B;  // <= 2 n_kv_ctas, checked above
+        if ((st = preprocess()) != FA_OK) return st;
         bwd_pair_kernel<<<(unsigned)n_pair_ctas, 512, sizeof(BwdPairSmem), stream>>>(tq, tq64, tk, tv, tdo, tdo64, tdk,
                                                                                       tdv, p, n_kv_pairs);
         if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
       } else if (s.f16) {
-        static bool attr_h = false;
-        if ((st = set_smem(bwd_fused_kernel<true>, (int)sizeof(BwdFusedSmem), &attr_h)) != FA_OK) return st;
+        if ((st = set_smem_once(bwd_fused_kernel<true>, (int)sizeof(BwdFusedSmem), g_attr_fused_f16)) != FA_OK) return st;
+        if ((st = preprocess()) != FA_OK) return st;
         bwd_fused_kernel<true><<<(unsigned)n_kv_ctas, 512, sizeof(BwdFusedSmem), stream>>>(tq, tk, tv, tdo, tdk, tdv, p,
                                                                                           n_kv_tiles);
         if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
       } else {
-        static bool attr_f = false;
-        if ((st = set_smem(bwd_fused_kernel<false>, (int)sizeof(BwdFusedSmem), &attr_f)) != FA_OK) return st;
+        if ((st = set_smem_once(bwd_fused_kernel<false>, (int)sizeof(BwdFusedSmem), g_attr_fused_bf16)) != FA_OK) return st;
+        if ((st = preprocess()) != FA_OK) return st;
         bwd_fused_kernel<false><<<(unsigned)n_kv_ctas, 512, sizeof(BwdFusedSmem), stream>>>(tq, tk, tv, tdo, tdk, tdv, p,
                                                                                            n_kv_tiles);
         if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
       }
-      const size_t n8 = (size_t)s.B * s.Sq * s.H * D / 8;
-      const size_t blocks = (n8 + 255) / 256;
-      if (blocks > 0x7fffffffull) return FA_ERR_UNSUPPORTED;
       auto conv = s.f16 ? bwd_convert_dq_chunked_kernel<true> : bwd_convert_dq_chunked_kernel<false>;
-      conv<<<(unsigned)blocks, 256, 0, stream>>>(dq_acc, static_cast<__nv_bfloat16*>(dq), n8, s.scale, s.H, s.Sq,
+      conv<<<(unsigned)conv_blocks, 256, 0, stream>>>(dq_acc, static_cast<__nv_bfloat16*>(dq), n8, s.scale, s.H, s.Sq,
                                                  w.sq_pad);
       return cudaGetLastError() == cudaSuccess ? FA_OK : FA_ERR_CUDA;
     }
   }
   // 2a. dK, dV;  2b. dQ
-  if (s.f16) return bwd_split_launch<D, true>(tq, tk, tv, tdo, tdq, tdk, tdv, p, n_kv_tiles, n_q_tiles, stream);
-  return bwd_split_launch<D, false>(tq, tk, tv, tdo, tdq, tdk, tdv, p, n_kv_tiles, n_q_tiles, stream);
+  if (s.f16) return bwd_split_launch<D, true>(tq, tk, tv, tdo, tdq, tdk, tdv, p, n_kv_tiles, n_q_tiles, preprocess, stream);
+  return bwd_split_launch<D, false>(tq, tk, tv, tdo, tdq, tdk, tdv, p, n_kv_tiles, n_q_tiles, preprocess, stream);
 }
 
 // ---------------------------------------------------------------- variable-length batches
@@ -210,18 +205,23 @@ int bwd_varlen_launch(const void* q, const void* k, const void* v, const void* o
   if ((st = encode_bshd_map(&tdk, dk, 1, total_k, s.Hkv, D, 64, 128, bf16, 2, sw)) != FA_OK) return st;
   if ((st = encode_bshd_map(&tdv, dv, 1, total_k, s.Hkv, D, 64, 128, bf16, 2, sw)) != FA_OK) return st;
 
+  // Every size check and per-device set-up comes before the first launch.
+  const long long pre_blocks = ((long long)s.H * tp + 15) / 16;
+  const int n_kv_tiles = (s.Sk + 127) / 128;
+  const long long n_ctas = (long long)n_kv_tiles * s.Hkv * s.B;
+  const size_t n8 = (size_t)total_q * s.H * D / 8;
+  const size_t conv_blocks = (n8 + 255) / 256;
+  if (pre_blocks > 0x7fffffffll || n_ctas > 0x7fffffffll || conv_blocks > 0x7fffffffull) return FA_ERR_UNSUPPORTED;
+  st = s.f16 ? set_smem_once(bwd_fused_kernel<true>, (int)sizeof(BwdFusedSmem), g_attr_fused_f16)
+             : set_smem_once(bwd_fused_kernel<false>, (int)sizeof(BwdFusedSmem), g_attr_fused_bf16);
+  if (st != FA_OK) return st;
+
   varlen_pad_offsets_kernel<<<1, 32, 0, stream>>>(cu_q, s.B, pad_off);
   if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
-  {
-    const long long rows = (long long)s.H * tp;
-    const long long blocks = (rows + 15) / 16;
-    if (blocks > 0x7fffffffll) return FA_ERR_UNSUPPORTED;
-    auto pre = s.f16 ? bwd_preprocess_varlen_kernel<true> : bwd_preprocess_varlen_kernel<false>;
-    pre<<<(unsigned)blocks, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(o),
-                                              static_cast<const __nv_bfloat16*>(d_o), lse, delta, lse2, dq_acc, cu_q,
-                                              pad_off, s.B, s.H, total_q, tp);
-    if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
-  }
+  auto pre = s.f16 ? bwd_preprocess_varlen_kernel<true> : bwd_preprocess_varlen_kernel<false>;
+  pre<<<(unsigned)pre_blocks, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(o), static_cast<const __nv_bfloat16*>(d_o),
+                                                lse, delta, lse2, dq_acc, cu_q, pad_off, s.B, s.H, total_q, tp);
+  if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
   BwdParams p;
   p.dq_acc = dq_acc;
   p.lse2 = lse2;
@@ -230,32 +230,24 @@ int bwd_varlen_launch(const void* q, const void* k, const void* v, const void* o
   p.scale = s.scale;
   p.scale_log2 = s.scale * kLog2e;
   p.causal = s.causal;
+  p.epoch = next_launch_epoch();
   p.cu_q = cu_q;
   p.cu_k = cu_k;
   p.pad_off = pad_off;
   p.total_pad = tp;
   p.dk = static_cast<__nv_bfloat16*>(dk);
   p.dv = static_cast<__nv_bfloat16*>(dv);
-  const int n_kv_tiles = (s.Sk + 127) / 128;
-  const long long n_ctas = (long long)n_kv_tiles * s.Hkv * s.B;
-  if (n_ctas > 0x7fffffffll) return FA_ERR_UNSUPPORTED;
-  static bool attr_f = false, attr_h = false;
   if (s.f16) {
-    if ((st = set_smem(bwd_fused_kernel<true>, (int)sizeof(BwdFusedSmem), &attr_h)) != FA_OK) return st;
     bwd_fused_kernel<true><<<(unsigned)n_ctas, 512, sizeof(BwdFusedSmem), stream>>>(tq, tk, tv, tdo, tdk, tdv, p,
                                                                                    n_kv_tiles);
   } else {
-    if ((st = set_smem(bwd_fused_kernel<false>, (int)sizeof(BwdFusedSmem), &attr_f)) != FA_OK) return st;
     bwd_fused_kernel<false><<<(unsigned)n_ctas, 512, sizeof(BwdFusedSmem), stream>>>(tq, tk, tv, tdo, tdk, tdv, p,
                                                                                     n_kv_tiles);
   }
   if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
-  const size_t n8 = (size_t)total_q * s.H * D / 8;
-  const size_t blocks = (n8 + 255) / 256;
-  if (blocks > 0x7fffffffull) return FA_ERR_UNSUPPORTED;
   auto conv = s.f16 ? bwd_convert_dq_varlen_kernel<true> : bwd_convert_dq_varlen_kernel<false>;
-  conv<<<(unsigned)blocks, 256, 0, stream>>>(dq_acc, static_cast<__nv_bfloat16*>(dq), n8, s.scale, cu_q, pad_off, s.B,
-                                             s.H, tp);
+  conv<<<(unsigned)conv_blocks, 256, 0, stream>>>(dq_acc, static_cast<__nv_bfloat16*>(dq), n8, s.scale, cu_q, pad_off,
+                                                  s.B, s.H, tp);
   return cudaGetLastError() == cudaSuccess ? FA_OK : FA_ERR_CUDA;
 }
 
@@ -267,8 +259,3 @@ int bwd_launch(const void* q, const void* k, const void* v, const void* o, const
 
 }  // namespace fa
 
-#ifdef FA_PROFILE_PHASES
-extern "C" int fa_debug_pair_trace(long long* host_out) {
-  return (int)cudaMemcpyFromSymbol(host_out, fa::g_pair_trace, sizeof(long long) * 128);
-}
-#endif

@@ -32,7 +32,7 @@ struct BwdFusedSmem {
   uint64_t q_full[2], q_empty[2], do_full, do_empty;
   uint64_t s_full, p_ready, dp_full, dst_ready, ds_ready, dq_full, dq_drained, acc_full, out_staged;
   uint32_t tmem_base;
-  int abort_flag;
+  WaitCtl ctl;  // abort flag and launch epoch, read by every bounded wait
 };
 
 // dQ accumulator element (b, h, q, d) in the chunked layout the bulk reductions use.
@@ -72,7 +72,7 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   using Smem = BwdFusedSmem;
   Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
   if ((smem_u32(smem_raw) & 1023u) != 0) {
-    if (threadIdx.x == 0) atomicExch(&g_device_status, 5);
+    if (threadIdx.x == 0) record_device_status(5, __LINE__, p.epoch);
     return;
   }
   constexpr int kRegions = 2;
@@ -83,7 +83,7 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   constexpr uint32_t kColR0 = 0, kColR1 = 128, kColDv = 256, kColDk = 384;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  volatile int* abort_flag = &sm.abort_flag;
+  volatile int* abort_flag = &sm.ctl.abort_flag;
 
   const int n_tile = blockIdx.x % n_kv_tiles;
   const int hk = (blockIdx.x / n_kv_tiles) % p.Hkv;
@@ -117,7 +117,8 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int q_rot = iters_per_head > 0 ? n_tile % iters_per_head : 0;
 
   if (tid == 0) {
-    sm.abort_flag = 0;
+    sm.ctl.abort_flag = 0;
+    sm.ctl.launch_epoch = (int)p.epoch;
     mbar_init(&sm.kv_full, 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sm.q_full[s], 1);

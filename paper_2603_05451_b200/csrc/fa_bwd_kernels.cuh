@@ -20,7 +20,7 @@
 #pragma once
 
 #include "fa_common.cuh"
-#include "fa_fwd_simple.cuh"  // kLog2e
+#include "fa_fwd_params.cuh"  // kLog2e
 #include "ptx.cuh"
 
 namespace fa {
@@ -32,6 +32,7 @@ struct BwdParams {
   int B, H, Hkv, Sq, Sk, Sq_pad;
   float scale, scale_log2;
   int causal;
+  unsigned epoch;  // identifies this launch in the device status word (bounded waits)
   // Variable-length batches (fused kernel only; null / 0 otherwise): sequence b owns query tokens
   // [cu_q[b], cu_q[b+1]) and key tokens [cu_k[b], cu_k[b+1]) of the packed tensors; in the workspace
   // arrays (accumulator, lse2, delta: [H, total_pad, ...]) its rows start at pad_off[b], a multiple

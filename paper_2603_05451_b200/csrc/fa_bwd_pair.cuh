@@ -48,25 +48,10 @@ struct BwdPairSmem {
   uint64_t ds_in;                          // local: the other CTA's half of dS^T has landed in `ds`
   uint64_t out_staged;                     // local
   uint32_t tmem_base;
-  int abort_flag;
+  WaitCtl ctl;  // abort flag and launch epoch, read by every bounded wait
 };
 static_assert(sizeof(BwdPairSmem) <= 227 * 1024, "pair kernel shared memory");
 
-#ifdef FA_PROFILE_PHASES
-// Debug timeline (global nanosecond timer) of iterations [8, 12) of pair 0: [iteration][event].
-__device__ long long g_pair_trace[4 * 32];
-__device__ __forceinline__ long long pair_now() {
-  long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-#define FA_PTRACE(id, it)                                                                          \
-  do {                                                                                             \
-    if (blockIdx.x < 2 && (it) >= 8 && (it) < 12) g_pair_trace[((it) - 8) * 32 + (id)] = pair_now(); \
-  } while (0)
-#else
-#define FA_PTRACE(id, it)
-#endif
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(512, 1)
 bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_q64,
@@ -79,7 +64,7 @@ bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   using Smem = BwdPairSmem;
   Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
   if ((smem_u32(smem_raw) & 1023u) != 0) {  // same in both CTAs of a pair, so both leave
-    if (threadIdx.x == 0) atomicExch(&g_device_status, 5);
+    if (threadIdx.x == 0) record_device_status(5, __LINE__, p.epoch);
     return;
   }
   constexpr int kRegionBytes = 128 * 128;  // [128 rows][64 bf16]
@@ -93,7 +78,7 @@ bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   constexpr uint32_t kColR0 = 0, kColR1 = 128, kColDq = 160, kColDv = 256, kColDk = 384;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  volatile int* abort_flag = &sm.abort_flag;
+  volatile int* abort_flag = &sm.ctl.abort_flag;
   const uint32_t rank = cluster_cta_rank();
   const bool leader = rank == 0;
 
@@ -113,7 +98,8 @@ bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const int q_rot = iters_per_head > 0 ? pair % iters_per_head : 0;
 
   if (tid == 0) {
-    sm.abort_flag = 0;
+    sm.ctl.abort_flag = 0;
+    sm.ctl.launch_epoch = (int)p.epoch;
     mbar_init(&sm.kv_full, 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sm.qr_full[s], 1);
@@ -171,7 +157,6 @@ bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const int q0 = i * 128 + wg * 64;
       ok = __all_sync(0xffffffffu, mbar_wait(&sm.s_full, it & 1, abort_flag, __LINE__));
       if (!ok) break;
-      if (warp == 0 && lane == 0) FA_PTRACE(0 + 4 * rank, it);
       ok = __all_sync(0xffffffffu, mbar_wait(&sm.stat_full[stage], (it >> 1) & 1, abort_flag, __LINE__));
       if (!ok) break;
       tc_fence_after();
@@ -205,17 +190,14 @@ bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(bar_p_ready);
-      if (warp == 0 && lane == 0) FA_PTRACE(1 + 4 * rank, it);
 
       ok = __all_sync(0xffffffffu, mbar_wait(&sm.dp_full, it & 1, abort_flag, __LINE__));
       if (!ok) break;
-      if (warp == 0 && lane == 0) FA_PTRACE(2 + 4 * rank, it);
       tc_fence_after();
       uint32_t dp[2][32];
       tmem_ld32(dp_addr, dp[0]);
       tmem_ld32(dp_addr + 32, dp[1]);
       tmem_wait_ld();
-      if (warp == 0 && lane == 0) FA_PTRACE(15 + 12 * rank, it);
       const float4* dl4 =reinterpret_cast<const float4*>(&sm.delta[stage][wg * 64]);
 #pragma unroll
       for (int h2 = 0; h2 < 2; ++h2) {
@@ -230,7 +212,6 @@ bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           pk[g * 2] = pack_bf16x2(d0, d1);
           pk[g * 2 + 1] = pack_bf16x2(d2, d3);
         }
-        if (warp == 0 && lane == 0 && rank == 0) FA_PTRACE(28 + 2 * h2, it);
         tmem_st16(dp_addr + wg * 32 + h2 * 16, pk);
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
@@ -241,17 +222,12 @@ bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           if (ds_is_local) *reinterpret_cast<uint4*>(ds_row_local + off) = v4;
           else st_async_v4(ds_row + off, v4, bar_ds_in_peer);
         }
-        if (warp == 0 && lane == 0 && rank == 0) FA_PTRACE(29 + 2 * h2, it);
       }
-      if (warp == 0 && lane == 0) FA_PTRACE(12 + 12 * rank, it);
       tmem_wait_st();
       tc_fence_before();
-      if (warp == 0 && lane == 0) FA_PTRACE(13 + 12 * rank, it);
       if (ds_is_local) fence_proxy_async_smem();
       __syncwarp();
-      if (warp == 0 && lane == 0) FA_PTRACE(14 + 12 * rank, it);
       if (lane == 0) mbar_arrive_cluster(bar_ds_ready);
-      if (warp == 0 && lane == 0) FA_PTRACE(3 + 4 * rank, it);
     }
 
     // ---- epilogue: dV and dK * scale of this CTA's key rows -> bf16 -> shared memory (swizzled) -> TMA store
@@ -321,7 +297,6 @@ bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const int i = i_first + (it % iters_per_head + q_rot) % iters_per_head;
       ok = __all_sync(0xffffffffu, mbar_wait(&sm.dq_full, it & 1, abort_flag, __LINE__));
       if (!ok) break;
-      if (warp == 8 && lane == 0) FA_PTRACE(8 + 2 * rank, it);
       tc_fence_after();
       uint32_t v[2][32];
       tmem_ld32(addr, v[0]);
@@ -331,7 +306,6 @@ bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(bar_dq_drained);
-      if (warp == 8 && lane == 0) FA_PTRACE(9 + 2 * rank, it);
       float* dst = p.dq_acc +
                    ((((size_t)b * p.H + h) * (p.Sq_pad / 32) + (size_t)i * 4 + 2 * (w >> 1)) * 4 + d_chunk) * 1024;
 #pragma unroll
@@ -409,27 +383,21 @@ bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           if (!(ok = wait_bar(&sm.do_full, it & 1, __LINE__))) break;
           if (it > 0 && !(ok = wait_bar(&sm.dq_drained, (it - 1) & 1, __LINE__))) break;
           tc_fence_after();
-          if (lane == 0) FA_PTRACE(16, it);  // do_full and dq_drained seen
           ss_kmajor(kColR1, v_lo, dor_lo);  // dP^T(it)
           commit(&sm.dp_full);
-          if (lane == 0) FA_PTRACE(17, it);
           if (!(ok = wait_bar(&sm.p_ready, it & 1, __LINE__))) break;
           tc_fence_after();
-          if (lane == 0) FA_PTRACE(18, it);  // p_ready seen
           ts_acc(kColDv, kColR0, 64, doc_lo, it > 0 ? 1u : 0u);  // dV += P^T dO
           commit(&sm.do_empty);
-          if (lane == 0) FA_PTRACE(19, it);
           if (it + 1 < n_iter) {
             if (!(ok = wait_bar(&sm.qr_full[stage ^ 1], ((it + 1) >> 1) & 1, __LINE__))) break;
             ss_kmajor(kColR0, k_lo, qr_lo0 + (stage ^ 1) * kQrStageStep);  // S^T(it + 1)
             commit(&sm.s_full);
             commit(&sm.qr_empty[stage ^ 1]);
           }
-          if (lane == 0) FA_PTRACE(20, it);  // next S^T issued
           if (!(ok = wait_bar(&sm.ds_ready, it & 1, __LINE__))) break;
           if (!(ok = wait_bar(&sm.ds_in, it & 1, __LINE__))) break;
           tc_fence_after();
-          if (lane == 0) FA_PTRACE(21, it);  // dS^T complete in both CTAs
           // dQ^T first: its drain and the hand-back of the region then overlap with the dK product
           if (elect_one()) {
             if (it + 1 < n_iter) mbar_expect_tx(&sm.ds_in, Smem::kHalfBytes);
@@ -443,7 +411,6 @@ bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           if (!(ok = wait_bar(&sm.qc_full, it & 1, __LINE__))) break;
           ts_acc(kColDk, kColR1, 96, qc_lo, it > 0 ? 1u : 0u);  // dK += dS^T Q
           commit(&sm.qc_empty);
-          if (lane == 0) FA_PTRACE(22, it);
         }
         if (ok) commit(&sm.acc_full);
       } while (false);

@@ -36,7 +36,7 @@ struct BwdDkdvSmem {
   uint64_t q_full[2], do_full[2], stage_empty[2];
   uint64_t s_full, p_ready, dp_full, ds_ready, acc_full, out_staged;
   uint32_t tmem_base;
-  int abort_flag;
+  WaitCtl ctl;  // abort flag and launch epoch, read by every bounded wait
 };
 
 template <int D, bool kF16 = false>
@@ -49,7 +49,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   using Smem = BwdDkdvSmem<D>;
   Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
   if ((smem_u32(smem_raw) & 1023u) != 0) {
-    if (threadIdx.x == 0) atomicExch(&g_device_status, 5);
+    if (threadIdx.x == 0) record_device_status(5, __LINE__, p.epoch);
     return;
   }
   constexpr int kRegions = D / 64;
@@ -59,7 +59,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   constexpr uint32_t kColR0 = 0, kColR1 = 128, kColDv = 256, kColDk = 384;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  volatile int* abort_flag = &sm.abort_flag;
+  volatile int* abort_flag = &sm.ctl.abort_flag;
 
   // work decode: key tiles ascending (with a causal mask the first tile sees the most queries), kv heads, batches
   const int n_tile = blockIdx.x % n_kv_tiles;
@@ -75,7 +75,8 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const int n_iter = iters_per_head * group;
 
   if (tid == 0) {
-    sm.abort_flag = 0;
+    sm.ctl.abort_flag = 0;
+    sm.ctl.launch_epoch = (int)p.epoch;
     mbar_init(&sm.kv_full, 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sm.q_full[s], 1);
@@ -341,7 +342,7 @@ struct BwdDqSmem {
   uint64_t kv_full[2], kv_empty[2];
   uint64_t s_full, s_free, dp_full[2], ds_ready, acc_full, out_staged;  // dp_full: one per ping-pong region
   uint32_t tmem_base;
-  int abort_flag;
+  WaitCtl ctl;  // abort flag and launch epoch, read by every bounded wait
 };
 
 template <int D, bool kF16 = false>
@@ -353,7 +354,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
   using Smem = BwdDqSmem<D>;
   Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
   if ((smem_u32(smem_raw) & 1023u) != 0) {
-    if (threadIdx.x == 0) atomicExch(&g_device_status, 5);
+    if (threadIdx.x == 0) record_device_status(5, __LINE__, p.epoch);
     return;
   }
   constexpr int kRegions = D / 64;
@@ -364,7 +365,7 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
   constexpr uint32_t kColS = 0, kColDp0 = 128, kColDq = 384;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  volatile int* abort_flag = &sm.abort_flag;
+  volatile int* abort_flag = &sm.ctl.abort_flag;
 
   // work decode: batches outermost, query tiles from the LAST one down (longest first under a causal mask), heads fastest
   const int h = blockIdx.x % p.H;
@@ -383,7 +384,8 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
   }
 
   if (tid == 0) {
-    sm.abort_flag = 0;
+    sm.ctl.abort_flag = 0;
+    sm.ctl.launch_epoch = (int)p.epoch;
     mbar_init(&sm.q_full, 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sm.kv_full[s], 1);

@@ -8,6 +8,8 @@
 #include <stdint.h>
 #include <stddef.h>
 
+#include <atomic>
+
 #include "../../include/fa.h"
 
 namespace fa {
@@ -40,7 +42,35 @@ int bwd_varlen_launch(const void* q, const void* k, const void* v, const void* o
                       void* dq, void* dk, void* dv, const int* cu_q, const int* cu_k, int total_q, int total_k,
                       const Shape& s, void* workspace, cudaStream_t stream);
 
-// Reads an integer option from the environment once per process (`deflt` when unset).
+// Reads an integer option from the environment (`deflt` when unset).
 int env_int(const char* name, int deflt);
+
+// A fresh identifier for one entry-point call; kernels store it beside a recorded device-side
+// failure so that only the blocks of the failing launch give up early.
+unsigned next_launch_epoch();
+
+// State that CUDA keeps per device (function attributes, the architecture check) is cached per
+// device ordinal: one flag per device, set after the first successful set-up on that device.
+constexpr int kMaxDevices = 64;
+struct PerDeviceFlag {
+  std::atomic<int> value[kMaxDevices];  // zero-initialised (static storage)
+  bool test(int dev) const { return dev >= 0 && dev < kMaxDevices && value[dev].load(std::memory_order_acquire) != 0; }
+  void set(int dev, int v = 1) {
+    if (dev >= 0 && dev < kMaxDevices) value[dev].store(v, std::memory_order_release);
+  }
+  int get(int dev) const { return dev >= 0 && dev < kMaxDevices ? value[dev].load(std::memory_order_acquire) : 0; }
+};
+
+// Raises the dynamic shared-memory limit of `kernel` to `bytes` on the current device, once per device.
+template <typename Kernel>
+int set_smem_once(Kernel kernel, int bytes, PerDeviceFlag& done) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FA_ERR_CUDA;
+  if (done.test(dev)) return FA_OK;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess)
+    return FA_ERR_CUDA;
+  done.set(dev);
+  return FA_OK;
+}
 
 }  // namespace fa

@@ -1,7 +1,6 @@
 // Forward-pass launch code: builds the tensor maps and launches the kernel.
 #include "fa_common.cuh"
 #include "fa_fwd_pipe.cuh"
-#include "fa_fwd_simple.cuh"
 
 namespace fa {
 
@@ -17,6 +16,9 @@ static int make_maps(CUtensorMap* tq, CUtensorMap* tk, CUtensorMap* tv, CUtensor
   return FA_OK;
 }
 
+// Default share of exponentials computed on the FMA pipe, per head dimension (of every 8).
+constexpr int kDefaultEmuPer8D64 = 0, kDefaultEmuPer8D128 = 0;
+
 static FwdParams make_params(void* o, float* lse, const Shape& s) {
   FwdParams p;
   p.o = static_cast<__nv_bfloat16*>(o);
@@ -31,7 +33,7 @@ static FwdParams make_params(void* o, float* lse, const Shape& s) {
   }();
   p.tau = tau;
   p.causal = s.causal;
-  p.dbg = nullptr;
+  p.epoch = next_launch_epoch();
   // Sections of heads whose K and V (2 * Sk * (Dqk + Dv) bytes per key/value head; s.D stands for both
   // dimensions here, close enough for (192,128)) stay within a quarter of the 126 MB L2, so that the
   // blocks in flight re-read them from L2 and not from memory.  FA_FWD_SECTION_MB (read once) overrides
@@ -50,52 +52,29 @@ static FwdParams make_params(void* o, float* lse, const Shape& s) {
   return p;
 }
 
-template <int D>
-static int launch_simple(const void* q, const void* k, const void* v, void* o, float* lse, const Shape& s,
-                         cudaStream_t stream) {
-  CUtensorMap tq, tk, tv;
-  int st = make_maps(&tq, &tk, &tv, nullptr, q, k, v, o, s);
-  if (st != FA_OK) return st;
-  FwdParams p = make_params(o, lse, s);
-#ifdef FA_DEBUG_DUMP
-  p.dbg = reinterpret_cast<float*>((uintptr_t)strtoull(getenv("FA_DBG_PTR") ? getenv("FA_DBG_PTR") : "0", nullptr, 0));
-#endif
-  const int smem = sizeof(FwdSimpleSmem<D>) + 1024;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(fwd_simple_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
-      return FA_ERR_CUDA;
-    attr_set = true;
-  }
-  dim3 grid((s.Sq + 127) / 128, s.H, s.B);
-  if (grid.y > 65535u || grid.z > 65535u) return FA_ERR_UNSUPPORTED;
-  fwd_simple_kernel<D><<<grid, 128, smem, stream>>>(tq, tk, tv, p);
-  return cudaGetLastError() == cudaSuccess ? FA_OK : FA_ERR_CUDA;
-}
-
-template <int D, int kEmuPer8, bool kSer = false, bool kF16 = false>
-static int launch_pipe(const void* q, const void* k, const void* v, void* o, float* lse, const Shape& s,
-                       cudaStream_t stream) {
-  CUtensorMap tq, tk, tv, to;
-  int st = make_maps(&tq, &tk, &tv, &to, q, k, v, o, s);
-  if (st != FA_OK) return st;
-  FwdParams p = make_params(o, lse, s);
-#ifdef FA_PROFILE_PHASES
-  p.dbg = reinterpret_cast<float*>((uintptr_t)strtoull(getenv("FA_DBG_PTR") ? getenv("FA_DBG_PTR") : "0", nullptr, 0));
-#endif
-  const int smem = sizeof(FwdPipeSmem<D, D>);
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(fwd_pipe_kernel<D, D, kEmuPer8, kSer, kF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
-        cudaSuccess)
-      return FA_ERR_CUDA;
-    attr_set = true;
-  }
+// One launch of the pipelined kernel: tensor maps, parameters, shared-memory opt-in (once per device).
+template <int DQK, int DV, int kEmuPer8, bool kF16>
+static int launch_pipe(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                       const FwdParams& p, const Shape& s, cudaStream_t stream) {
+  static PerDeviceFlag attr_set;
+  constexpr int smem = (int)sizeof(FwdPipeSmem<DQK, DV>);
+  auto kernel = fwd_pipe_kernel<DQK, DV, kEmuPer8, kF16>;
   const int n_mblocks = (s.Sq + 255) / 256;
   const long long n_ctas = (long long)s.B * s.H * n_mblocks;
   if (n_ctas > 0x7fffffffll) return FA_ERR_UNSUPPORTED;
-  fwd_pipe_kernel<D, D, kEmuPer8, kSer, kF16><<<(unsigned)n_ctas, 512, smem, stream>>>(tq, tk, tv, to, p, n_mblocks);
+  int st = set_smem_once(kernel, smem, attr_set);
+  if (st != FA_OK) return st;
+  kernel<<<(unsigned)n_ctas, 512, smem, stream>>>(tq, tk, tv, to, p, n_mblocks);
   return cudaGetLastError() == cudaSuccess ? FA_OK : FA_ERR_CUDA;
+}
+
+template <int D, int kEmuPer8, bool kF16 = false>
+static int launch_dense(const void* q, const void* k, const void* v, void* o, float* lse, const Shape& s,
+                        cudaStream_t stream) {
+  CUtensorMap tq, tk, tv, to;
+  int st = make_maps(&tq, &tk, &tv, &to, q, k, v, o, s);
+  if (st != FA_OK) return st;
+  return launch_pipe<D, D, kEmuPer8, kF16>(tq, tk, tv, to, make_params(o, lse, s), s, stream);
 }
 
 // Head dimensions (192, 128): s.D is the query/key dimension (192); values and output have 128.
@@ -109,52 +88,36 @@ int fwd_hd192_launch(const void* q, const void* k, const void* v, void* o, float
   if ((st = encode_bshd_map(&tk, k, s.B, s.Sk, s.Hkv, 192, 64, 128, bf16, 2, sw)) != FA_OK) return st;
   if ((st = encode_bshd_map(&tv, v, s.B, s.Sk, s.Hkv, 128, 64, 128, bf16, 2, sw)) != FA_OK) return st;
   if ((st = encode_bshd_map(&to, o, s.B, s.Sq, s.H, 128, 64, 128, bf16, 2, sw)) != FA_OK) return st;
-  FwdParams p = make_params(o, lse, s);
-  const int smem = sizeof(FwdPipeSmem<192, 128>);
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(fwd_pipe_kernel<192, 128, 0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
-      return FA_ERR_CUDA;
-    attr_set = true;
-  }
-  const int n_mblocks = (s.Sq + 255) / 256;
-  const long long n_ctas = (long long)s.B * s.H * n_mblocks;
-  if (n_ctas > 0x7fffffffll) return FA_ERR_UNSUPPORTED;
-  fwd_pipe_kernel<192, 128, 0, false><<<(unsigned)n_ctas, 512, smem, stream>>>(tq, tk, tv, to, p, n_mblocks);
-  return cudaGetLastError() == cudaSuccess ? FA_OK : FA_ERR_CUDA;
+  return launch_pipe<192, 128, 0, false>(tq, tk, tv, to, make_params(o, lse, s), s, stream);
+}
+
+// How many of every 8 exponentials use the software 2^x (Section 3.1.3).  The default is chosen per
+// head dimension; FA_EMU_PER8 = 0..3 (read once per process) overrides it for both.
+static int emu_per8(int D) {
+  static const int forced = env_int("FA_EMU_PER8", -1);
+  if (forced >= 0) return forced > 3 ? 3 : forced;
+  return D == 64 ? kDefaultEmuPer8D64 : kDefaultEmuPer8D128;
 }
 
 int fwd_launch(const void* q, const void* k, const void* v, void* o, float* lse, const Shape& s, cudaStream_t stream) {
-  // Experiment switches, read once: FA_FWD_IMPL=simple picks the straight-line kernel;
-  // FA_EMU_PER8 = how many of every 8 exponentials use the software 2^x (0, 1, 2 or 3).
-  static const int impl_simple = [] {
-    const char* e = getenv("FA_FWD_IMPL");
-    return (e && strcmp(e, "simple") == 0) ? 1 : 0;
-  }();
-  static const int emu = env_int("FA_EMU_PER8", 0);
-  // FA_SERIALISE_EXP=1: the two softmax warps of an SM sub-partition take turns on the exponential unit.
-  static const int ser = env_int("FA_SERIALISE_EXP", 0);
-  if (s.f16) {  // FP16 elements: the pipelined kernel without experiment switches
-    return s.D == 64 ? launch_pipe<64, 0, false, true>(q, k, v, o, lse, s, stream)
-                     : launch_pipe<128, 0, false, true>(q, k, v, o, lse, s, stream);
+  if (s.f16) {  // FP16 elements: MUFU exponentials only
+    return s.D == 64 ? launch_dense<64, 0, true>(q, k, v, o, lse, s, stream)
+                     : launch_dense<128, 0, true>(q, k, v, o, lse, s, stream);
   }
-  if (ser && !impl_simple && s.D == 128) return launch_pipe<128, 0, true>(q, k, v, o, lse, s, stream);
-  if (impl_simple) {
-    return s.D == 64 ? launch_simple<64>(q, k, v, o, lse, s, stream) : launch_simple<128>(q, k, v, o, lse, s, stream);
-  }
+  const int emu = emu_per8(s.D);
   if (s.D == 64) {
     switch (emu) {
-      case 1: return launch_pipe<64, 1>(q, k, v, o, lse, s, stream);
-      case 2: return launch_pipe<64, 2>(q, k, v, o, lse, s, stream);
-      case 3: return launch_pipe<64, 3>(q, k, v, o, lse, s, stream);
-      default: return launch_pipe<64, 0>(q, k, v, o, lse, s, stream);
+      case 1: return launch_dense<64, 1>(q, k, v, o, lse, s, stream);
+      case 2: return launch_dense<64, 2>(q, k, v, o, lse, s, stream);
+      case 3: return launch_dense<64, 3>(q, k, v, o, lse, s, stream);
+      default: return launch_dense<64, 0>(q, k, v, o, lse, s, stream);
     }
   }
   switch (emu) {
-    case 1: return launch_pipe<128, 1>(q, k, v, o, lse, s, stream);
-    case 2: return launch_pipe<128, 2>(q, k, v, o, lse, s, stream);
-    case 3: return launch_pipe<128, 3>(q, k, v, o, lse, s, stream);
-    default: return launch_pipe<128, 0>(q, k, v, o, lse, s, stream);
+    case 1: return launch_dense<128, 1>(q, k, v, o, lse, s, stream);
+    case 2: return launch_dense<128, 2>(q, k, v, o, lse, s, stream);
+    case 3: return launch_dense<128, 3>(q, k, v, o, lse, s, stream);
+    default: return launch_dense<128, 0>(q, k, v, o, lse, s, stream);
   }
 }
 
@@ -199,29 +162,12 @@ int fwd_varlen_launch(const void* q, const void* k, const void* v, void* o, floa
   p.cu_k = cu_k;
   p.order = order;
   p.total_q = total_q;
-  const int n_mblocks = (s.Sq + 255) / 256;
-  const long long n_ctas = (long long)s.B * s.H * n_mblocks;
-  if (n_ctas > 0x7fffffffll) return FA_ERR_UNSUPPORTED;
   CUtensorMap tq, tk, tv, to;
   int st = make_maps(&tq, &tk, &tv, &to, q, k, v, o, packed);
   if (st != FA_OK) return st;
-  auto launch = [&](auto kernel, int smem) {
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
-      return (int)FA_ERR_CUDA;
-    kernel<<<(unsigned)n_ctas, 512, smem, stream>>>(tq, tk, tv, to, p, n_mblocks);
-    return cudaGetLastError() == cudaSuccess ? (int)FA_OK : (int)FA_ERR_CUDA;
-  };
-  if (s.D == 64) return launch(fwd_pipe_kernel<64, 64, 0, false>, (int)sizeof(FwdPipeSmem<64, 64>));
-  return launch(fwd_pipe_kernel<128, 128, 0, false>, (int)sizeof(FwdPipeSmem<128, 128>));
+  if (s.D == 64) return launch_pipe<64, 64, 0, false>(tq, tk, tv, to, p, s, stream);
+  return launch_pipe<128, 128, 0, false>(tq, tk, tv, to, p, s, stream);
 }
 
 }  // namespace fa
 
-#ifdef FA_COUNT_RESCALES
-// Evidence build only: reads (and clears) the count of O rescales since the last call.
-extern "C" int fa_debug_rescale_count(unsigned long long* host_out) {
-  unsigned long long zero = 0;
-  if (cudaMemcpyFromSymbol(host_out, fa::g_rescale_count, sizeof(zero)) != cudaSuccess) return 3;
-  return cudaMemcpyToSymbol(fa::g_rescale_count, &zero, sizeof(zero)) == cudaSuccess ? 0 : 3;
-}
-#endif

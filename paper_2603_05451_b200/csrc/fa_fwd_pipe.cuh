@@ -10,20 +10,20 @@
 //               O_t += P_t V_j  (P read from tensor memory, V from shared memory)
 //   warp 13     TMA producer: Q tiles once, then K_j, V_j through an mbarrier ring
 //   warps 14-15 idle (they only donate registers)
-// Tensor memory (512 columns): S_0 [0,128) S_1 [128,256) O_0 [256,256+D) O_1 [384,384+D);
-// P_t (bf16, 64 columns) overlays the start of S_t.
+// Tensor memory (512 columns): one score buffer S [0,128) shared by both tiles, the 16-bit
+// probabilities P_0 [128,192) and P_1 [192,256), the accumulators O_0 [256,256+D) and O_1 [384,384+D).
 // Roles talk only through mbarriers with bounded waits; there is no CTA-wide barrier between
 // set-up and tear-down, so a role that gives up cannot strand another one.
 #pragma once
 
 #include "exp2_emu.cuh"
 #include "fa_common.cuh"
-#include "fa_fwd_simple.cuh"  // FwdParams and constants
+#include "fa_fwd_params.cuh"
 #include "ptx.cuh"
 
 namespace fa {
 
-// DQK = head dimension of queries and keys, DV = of values and the output (Section 4.1 benchmarks
+// DQK = head dimension of queries and keys, DV = of values and the output (Section 5 benchmarks
 // 64, 128 and the pair (192, 128)).  K blocks and V blocks travel through rings of their own:
 //   (128,128): 3 + 2 stages of 32 KiB   (64,64): 6 + 6 of 16 KiB   (192,128): 2 of 48 KiB + 1 of 32 KiB
 // which with the two Q tiles fills 224 KiB in every case.
@@ -49,28 +49,9 @@ struct FwdPipeSmem {
   uint64_t stat_full[2][4];  // softmax warp w of tile t -> correction warp w: scale[t][32w..] written
   uint64_t fin_full[2][4];   // softmax warp w of tile t -> correction warp w: inv_l[t][32w..] written (once)
   uint64_t o_staged[2];    // correction warps -> storing thread: O_t tile is in shared memory
-  uint64_t exp_done[2][4];  // softmax warp w of tile t finished the exponentials of a block (MUFU hand-over)
   uint32_t tmem_base;
-  int abort_flag;
-#ifdef FA_PROFILE_PHASES
-  long long trace[64];
-#endif
+  WaitCtl ctl;  // abort flag and launch epoch, read by every bounded wait
 };
-
-#ifdef FA_PROFILE_PHASES
-// Debug timeline: SM clock of event `id` (0..31) of block j in [8, 10), kept in shared memory.
-#define FA_TRACE(id, j)                                                                     \
-  do {                                                                                      \
-    if (blockIdx.x == 0 && (j) >= 8 && (j) < 10) sm.trace[((j) - 8) * 32 + (id)] = clock64(); \
-  } while (0)
-#else
-#define FA_TRACE(id, j)
-#endif
-
-#ifdef FA_COUNT_RESCALES
-// Evidence build only: how many times a correction warp rescaled its 32 rows of O (Section 3.1.4).
-__device__ unsigned long long g_rescale_count = 0;
-#endif
 
 struct FwdTile {
   int b, h, hk, m0;  // batch, query head, kv head, first query row of the CTA
@@ -102,7 +83,7 @@ __device__ __forceinline__ void softmax_exp_chunk(const uint32_t (&s)[32], uint3
 }
 
 // D: value / output head dimension; kF16: inputs and output are FP16 instead of BF16
-template <int DQK, int D, int kEmuPer8, bool kSerialiseExp, bool kF16 = false>
+template <int DQK, int D, int kEmuPer8, bool kF16 = false>
 __global__ void __launch_bounds__(512, 1)
 fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
@@ -111,7 +92,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   using Smem = FwdPipeSmem<DQK, D>;
   Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
   if ((smem_u32(smem_raw) & 1023u) != 0) {  // swizzled tiles need 1024-byte alignment; never seen, but checked
-    if (threadIdx.x == 0) atomicExch(&g_device_status, 5);
+    if (threadIdx.x == 0) record_device_status(5, __LINE__, p.epoch);
     return;
   }
   constexpr int kKStages = Smem::kKStages, kVStages = Smem::kVStages;
@@ -121,7 +102,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   constexpr uint32_t kIdescO = make_idesc(128, D, false, true, kF16);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  volatile int* abort_flag = &sm.abort_flag;
+  volatile int* abort_flag = &sm.ctl.abort_flag;
 
   // Work decode: batches outermost, then sections of heads whose K and V fit in L2 together, then
   // 256-row blocks from the LAST one down (longest causal tiles first, Section 3.3), the heads of the
@@ -165,13 +146,13 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const int n_blk_mine = (warp >> 2) == 1 ? n_blk[1] : n_blk[0];  // softmax warps: blocks of their tile
 
   if (tid == 0) {
-    sm.abort_flag = 0;
+    sm.ctl.abort_flag = 0;
+    sm.ctl.launch_epoch = (int)p.epoch;
     for (int t = 0; t < 2; ++t) {
       mbar_init(&sm.q_full[t], 1);
       mbar_init(&sm.s_full[t], 1);
       mbar_init(&sm.p_full[t], 8);  // 4 softmax warps + 4 correction warps
       mbar_init(&sm.p_last[t], 4);
-      for (int w = 0; w < 4; ++w) mbar_init(&sm.exp_done[t][w], 1);
       mbar_init(&sm.o_full[t], 1);
       mbar_init(&sm.o_staged[t], 4);
       for (int w = 0; w < 4; ++w) mbar_init(&sm.stat_full[t][w], 1);
@@ -219,24 +200,18 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int shift = Sk - Sq;
     const int row_limit = p.causal ? min(Sk - 1, row + shift) : Sk - 1;  // last visible key
     const int tile_first_limit = p.causal ? min(Sk - 1, tile.m0 + t * 128 + shift) : Sk - 1;
-    float m_run = -INFINITY, l_run = 0.0f;  // l_run: FP32 sum of the probabilities (LSE and the normalisation of O)
+    // l_run: FP32 sum of the unrounded probabilities (gives the LSE).  l_fix: what rounding to 16 bits
+    // added to the LARGEST probability of every block.  O is divided by l_run + l_fix: the products see
+    // the rounded probabilities, and in a row whose weight sits on one key the rounding of that one
+    // probability (up to 2^-9 relative when the running maximum is stale, Eq. 6) would otherwise show
+    // in O undiminished.  One exponential per row and block instead of a second sum over all elements.
+    float m_run = -INFINITY, l_run = 0.0f, l_fix = 0.0f;
     bool ok = true;
 
-#ifdef FA_PROFILE_PHASES
-    long long ph_acc[5] = {0, 0, 0, 0, 0};
-#define FA_MARK(i, a, b) ph_acc[i] += (b) - (a)
-#define FA_NOW(v) const long long v = clock64()
-#else
-#define FA_MARK(i, a, b)
-#define FA_NOW(v)
-#endif
     for (int j = 0; j < n_blk_mine; ++j) {
-      FA_NOW(c0);
       ok = __all_sync(0xffffffffu, mbar_wait(&sm.s_full[t], j & 1, abort_flag, __LINE__));
       if (!ok) break;
       tc_fence_after();
-      FA_NOW(c1);
-      if (lane == 0 && w == 0) FA_TRACE(0 + t, j);  // S seen by softmax
       uint32_t s[4][32];
       // The second half of the scores is fetched while the maxima of the first half are taken.
       tmem_ld32(s_addr, s[0]);
@@ -244,7 +219,6 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       tmem_wait_ld();
       tmem_ld32(s_addr + 64, s[2]);
       tmem_ld32(s_addr + 96, s[3]);
-      FA_NOW(c2);
 
       const int j0 = j * 128;
       const bool masked = j0 + 127 > tile_first_limit;  // block touches the mask of some row of this tile
@@ -271,7 +245,8 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           mx[3] = max3(mx[3], __uint_as_float(s[q4][i + 6]), __uint_as_float(s[q4][i + 7]));
         }
       }
-      const float m_new = fmaxf(max3(m_run, mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+      const float m_blk = fmaxf(max3(mx[0], mx[1], mx[2]), mx[3]);
+      const float m_new = fmaxf(m_run, m_blk);
       // Conditional rescale (Eq. 6): only when the maximum grew by more than tau in the base-2
       // domain; the decision is taken for the whole warp (Section 3.1.4, last sentence).
       const bool need = (m_new - m_run) * c > p.tau;
@@ -279,6 +254,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       if (__any_sync(0xffffffffu, need)) {
         f = (m_run == -INFINITY) ? 0.0f : ex2_approx((m_run - m_new) * c);
         l_run *= f;
+        l_fix *= f;
         m_run = m_new;
       }
       if (j > 0) {
@@ -293,65 +269,38 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       sm.scale[t][r_in_tile] = f;
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.stat_full[t][w]);
-      FA_NOW(c3);
-      if (lane == 0 && w == 0) FA_TRACE(2 + t, j);  // max done
 
-      // The two softmax warps that share an SM sub-partition take turns on its exponential unit
-      // (Section 3.1.2): tile 0's block j goes before tile 1's block j, then tile 0's block j + 1.
-      if (kSerialiseExp) {
-        const int other_n = t == 0 ? n_blk[1] : n_blk[0];
-        const int other_j = t == 0 ? j - 1 : j;
-        if (other_j >= 0 && other_j < other_n) {
-          ok = __all_sync(0xffffffffu, mbar_wait(&sm.exp_done[t ^ 1][w], other_j & 1, abort_flag, __LINE__));
-          if (!ok) break;
-        }
-      }
       const float neg_mc = (m_run == -INFINITY) ? 0.0f : -m_run * c;
+      {
+        const float p_top = ex2_approx(fmaf(m_blk, c, neg_mc));  // the block's largest probability, as computed below
+        l_fix += unpack2<kF16>(pack2<kF16>(p_top, 0.0f)).x - p_top;
+      }
       float2 sum2 = make_float2(0.0f, 0.0f);
 #pragma unroll
       for (int q4 = 0; q4 < 4; ++q4) {
         uint32_t pk[16];
         softmax_exp_chunk<D, kEmuPer8, kF16>(s[q4], pk, c, neg_mc, sum2);
         tmem_st16(p_addr + q4 * 16, pk);
-        if (lane == 0 && w == 0) FA_TRACE(16 + q4 * 2 + t, j);  // chunk q4 computed and its store issued
         if (q4 == 2) {
           // staged store: three quarters of P are enough to start O += P V
           tmem_wait_st();
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(&sm.p_full[t]);
-          if (lane == 0 && w == 0) FA_TRACE(4 + t, j);  // first 3/4 of P stored
         }
       }
-      if (kSerialiseExp) {
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.exp_done[t][w]);
-      }
       l_run += sum2.x + sum2.y;
-      FA_NOW(c4);
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.p_last[t]);
-      if (lane == 0 && w == 0) FA_TRACE(6 + t, j);  // all of P stored
-      FA_NOW(c5);
-      FA_MARK(0, c0, c1);
-      FA_MARK(1, c1, c2);
-      FA_MARK(2, c2, c3);
-      FA_MARK(3, c3, c4);
-      FA_MARK(4, c4, c5);
     }
-#ifdef FA_PROFILE_PHASES
-    if (p.dbg && lane == 0 && w == 0) {
-      for (int i = 0; i < 5; ++i) p.dbg[(blockIdx.x * 2 + t) * 8 + i] = (float)ph_acc[i] / max(1, n_blk_mine);
-    }
-#endif
 
     if (ok && valid[t]) {
       // Hand 1/l to the correction warp and write the LSE.  This uses a barrier of its own: nothing
       // orders it after the correction warp's wait for the last block's statistics, so an extra
       // phase of stat_full could run two phases ahead of a slow waiter and strand it.
-      sm.inv_l[t][r_in_tile] = l_run > 0.0f ? 1.0f / l_run : 0.0f;
+      sm.inv_l[t][r_in_tile] = l_run > 0.0f ? 1.0f / (l_run + l_fix) : 0.0f;
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.fin_full[t][w]);
       if (row < Sq) lse_rows[row] = l_run > 0.0f ? (m_run * c + log2f(l_run)) * kLn2 : -INFINITY;
@@ -369,9 +318,6 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (!ok) break;
         const float f = sm.scale[t][r_in_tile];
         if (j > 0 && __any_sync(0xffffffffu, f != 1.0f)) {
-#ifdef FA_COUNT_RESCALES
-          if (lane == 0) atomicAdd(&g_rescale_count, 1ull);  // one per (warp of 32 rows, block) that rescales O
-#endif
           ok = __all_sync(0xffffffffu, mbar_wait(&sm.o_full[t], (j - 1) & 1, abort_flag, __LINE__));
           if (!ok) break;
           tc_fence_after();
@@ -518,14 +464,10 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       auto do_pv = [&](int t, int j, int slot_v) -> bool {
         if (!wait_bar(&sm.p_full[t], j & 1)) return false;
         tc_fence_after();
-        FA_TRACE(8 + t, j);  // MMA thread saw p_full
         issue_pv(t, slot_v, j > 0 ? 1u : 0u, 0, 6);
-        FA_TRACE(10 + t, j);  // 6 PV MMAs issued
         if (!wait_bar(&sm.p_last[t], j & 1)) return false;
         tc_fence_after();
-        FA_TRACE(12 + t, j);  // MMA thread saw p_last
         issue_pv(t, slot_v, 1u, 6, 8);
-        FA_TRACE(14 + t, j);  // PV tail issued
         return true;
       };
       do {
@@ -606,9 +548,6 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
   tc_fence_before();
   __syncthreads();
-#ifdef FA_PROFILE_PHASES
-  if (p.dbg && blockIdx.x == 0 && tid < 64) reinterpret_cast<long long*>(p.dbg + gridDim.x * 24)[tid] = sm.trace[tid];
-#endif
   if (warp == 12) tmem_dealloc(tmem, 512);
 }
 

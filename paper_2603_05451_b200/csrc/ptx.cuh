@@ -12,8 +12,23 @@ namespace fa {
 
 // ------------------------------------------------------------------ device status
 // Written (never trapped on) when a bounded wait gives up; read by fa_last_device_status().
-// The library is built as one translation unit, so this definition is the only one.
-__device__ int g_device_status = 0;
+// Bits [0,8): status code, [8,32): source line of the wait that gave up, [32,64): epoch of the
+// launch that recorded it (every entry-point call gets a fresh epoch from the host).  The first
+// failure wins and stays until the host reads it.  The library is built as one translation unit,
+// so this definition is the only one.
+__device__ unsigned long long g_device_status = 0;
+
+__device__ __forceinline__ void record_device_status(int code, int site, unsigned epoch) {
+  atomicCAS(&g_device_status, 0ull,
+            ((unsigned long long)epoch << 32) | (unsigned long long)(unsigned)(code | (site << 8)));
+}
+// True when THIS launch (identified by its epoch) has already recorded a failure: its other
+// blocks should not each sit out their own limit.  A failure left behind by an earlier launch
+// does not count, so launches that follow an unread timeout still run normally.
+__device__ __forceinline__ bool launch_has_failed(unsigned epoch) {
+  const unsigned long long s = *reinterpret_cast<volatile unsigned long long*>(&g_device_status);
+  return (unsigned)s != 0u && (unsigned)(s >> 32) == epoch;
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -60,13 +75,16 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint64_t* bar, uint32_t parity
 
 // Wait limit in SM clock cycles (about half a second).  After it, the waiting thread records
 // FA_ERR_DEVICE_TIMEOUT, raises the CTA's abort flag and returns false; callers fall through to
-// the common exit, where tensor memory is released.  A recorded timeout also ends every other
-// unsatisfied wait on the device (the launch has failed as a whole; its remaining blocks should not
-// each sit out their own limit), until the host reads and clears the status word.
+// the common exit, where tensor memory is released.  A timeout recorded by the same launch also
+// ends every other unsatisfied wait of that launch.
 constexpr long long kWaitLimitCycles = 1ll << 30;
 
-// `site` (a source line) is kept in the status word's upper bits for diagnosis: the first wait that
-// gives up wins; the low byte is the status code.
+// `abort_flag` points at two consecutive ints in shared memory: the CTA's abort flag and the
+// epoch of the launch (WaitCtl below).  `site` (a source line) is kept in the status word for diagnosis.
+struct WaitCtl {
+  int abort_flag;
+  int launch_epoch;
+};
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int site = 0) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
@@ -74,10 +92,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 0x3ffu) == 0) {
-      if (*abort_flag || *reinterpret_cast<volatile int*>(&g_device_status) != 0) return false;
+      if (*abort_flag || launch_has_failed((unsigned)abort_flag[1])) return false;
       if (clock64() - t0 > kWaitLimitCycles) {
         *abort_flag = 1;
-        atomicCAS(&g_device_status, 0, 5 | (site << 8));
+        record_device_status(5, site, (unsigned)abort_flag[1]);
         return false;
       }
     }
@@ -358,10 +376,10 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity
   while (true) {
     if (mbar_try_wait_cluster(bar, parity)) return true;
     if ((++spins & 0x3ffu) == 0) {
-      if (*abort_flag || *reinterpret_cast<volatile int*>(&g_device_status) != 0) return false;
+      if (*abort_flag || launch_has_failed((unsigned)abort_flag[1])) return false;
       if (clock64() - t0 > kWaitLimitCycles) {
         *abort_flag = 1;
-        atomicCAS(&g_device_status, 0, 5 | (site << 8));
+        record_device_status(5, site, (unsigned)abort_flag[1]);
         return false;
       }
     }
