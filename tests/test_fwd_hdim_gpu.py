@@ -1,4 +1,4 @@
-"""Forward parity for head dimensions (192, 128) (Section 4.1's second forward workload): O and LSE
+"""Forward parity for head dimensions (192, 128) (Section 5's second forward workload): O and LSE
 from fa_fwd_hdim through the C ABI against the float64 oracle, element by element."""
 
 import numpy as np

@@ -1,0 +1,65 @@
+"""Forward parity for every kernel variant that an environment switch selects.
+
+The switches are read once per process, so each setting runs in a child interpreter that evaluates a
+list of shapes (several key blocks, ragged tails, causal, grouped heads, more queries than keys so
+that some rows see no key at all, both head dimensions, the x3 inputs that keep the conditional
+rescale busy) and prints its errors against the float64 oracle; the parent asserts the literal
+tolerances.
+
+  FA_EMU_PER8 = 1, 2, 3    that many of every 8 exponentials on the FMA pipe (Section 3.1.3)
+  FA_FWD_SECTION_MB = 0, 1  all heads in one launch section / sections of one key-value head (Section 3.3)
+"""
+
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+
+from tests.gpu_util import LSE_TOL, O_TOL
+
+pytestmark = pytest.mark.gpu
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+CHILD = r"""
+import json, sys
+sys.path.insert(0, %(root)r)
+from tests.test_fwd_gpu import _fwd_case
+# (B, H, Hkv, Sq, Sk, D, causal, multiplier of Q and K)
+cases = [(1, 1, 1, 128, 128, 64, False, 1.0), (2, 2, 2, 333, 333, 128, True, 1.0), (1, 3, 3, 300, 77, 128, True, 1.0),
+         (1, 2, 2, 1024, 1024, 128, False, 1.0), (1, 2, 2, 1024, 1024, 64, True, 1.0), (2, 8, 2, 640, 640, 128, True, 1.0),
+         (1, 4, 1, 200, 1100, 64, True, 1.0), (1, 2, 2, 1, 700, 128, False, 1.0), (1, 2, 2, 1536, 1536, 128, True, 3.0),
+         (1, 2, 2, 1536, 1536, 64, False, 3.0), (4, 4, 4, 2048, 2048, 128, True, 1.0)]
+out = []
+for idx, c in enumerate(cases):
+    eo, el = _fwd_case(*c[:7], seed=8100 + idx, mult=c[7], v_mult=1.0)
+    out.append([list(c), eo, el])
+print("RESULT " + json.dumps(out))
+"""
+
+
+@pytest.mark.parametrize("name,value", [("FA_EMU_PER8", "1"), ("FA_EMU_PER8", "2"), ("FA_EMU_PER8", "3"),
+                                        ("FA_FWD_SECTION_MB", "0"), ("FA_FWD_SECTION_MB", "1")])
+def test_forward_variants_match_the_oracle(name, value):
+    env = dict(os.environ)
+    env[name] = value
+    res = subprocess.run([sys.executable, "-c", CHILD % {"root": ROOT}], env=env, capture_output=True, text=True,
+                         timeout=900, cwd=ROOT)
+    assert res.returncode == 0, res.stderr[-2000:]
+    line = [l for l in res.stdout.splitlines() if l.startswith("RESULT ")][-1]
+    for case, eo, el in json.loads(line[len("RESULT "):]):
+        assert eo <= O_TOL and el <= LSE_TOL, (name, value, case, eo, el)
+
+
+def test_fa_log_names_the_wait_that_gave_up():
+    """FA_LOG=1: reading a recorded timeout prints the code and the source line of the wait."""
+    code = ("import sys; sys.path.insert(0, %r)\n"
+            "from paper_2603_05451_b200 import binding\n"
+            "binding.fa_selftest_unsatisfied_wait()\n"
+            "assert binding.fa_last_device_status() == 5\n") % ROOT
+    res = subprocess.run([sys.executable, "-c", code], env=dict(os.environ, FA_LOG="1"), capture_output=True, text=True,
+                         timeout=300, cwd=ROOT)
+    assert res.returncode == 0, res.stderr[-2000:]
+    assert "device-side wait expired (code 5, site" in res.stderr
