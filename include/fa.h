@@ -62,9 +62,9 @@ int fa_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
 
 /*
  * Bytes of scratch fa_bwd needs for these sizes: two FP32 row vectors [B, H, Sq_padded] (row dot
- * products of dO and O, and the log-sum-exp in base 2) plus, on the default D = 128 path, an FP32
- * dQ accumulator of B * H * Sq_padded * D elements (Sq_padded = Sq rounded up to 128).  Returns 0
- * for unsupported sizes.  Host-only; launches nothing.
+ * products of dO and O, and the log-sum-exp in base 2) plus an FP32 dQ accumulator of
+ * B * H * Sq_padded * D elements (Sq_padded = Sq rounded up to 128).  Returns 0 for unsupported
+ * sizes.  Host-only; launches nothing.
  */
 size_t fa_bwd_workspace_bytes(int B, int H, int Hkv, int Sq, int Sk, int D);
 
@@ -136,10 +136,10 @@ int fa_varlen_lpt_order(const int* cu_seqlens_q, const int* cu_seqlens_k, int ba
  * dq, dk, dv (bfloat16; not accumulated into).  `workspace` is caller-owned device scratch of
  * at least fa_bwd_workspace_bytes(...) bytes, 256-byte aligned; its contents on entry are
  * ignored and on return are unspecified.  Three kernel launches on `stream`.
- * D = 128 (default path): dq is summed across key/value tiles with floating-point reductions
- * whose order is not fixed, so dq is not bit-reproducible; dk and dv are.  D = 64, and every D
- * when the environment variable FA_BWD_IMPL=split is set before the first call: a
- * reduction-free two-kernel path whose dq, dk and dv are all bit-reproducible (slower at D = 128).
+ * Default path (D = 64 and 128): dq is summed across key/value tiles with floating-point reductions
+ * whose order is not fixed, so dq is not bit-reproducible; dk and dv are.  When the environment
+ * variable FA_BWD_IMPL=split is set before the first call: a reduction-free two-kernel path whose
+ * dq, dk and dv are all bit-reproducible (slower; it is what fa_bwd_deterministic runs).
  * FA_BWD_IMPL=pair (D = 128) runs the default path's main kernel on clusters of two thread blocks
  * (Section 3.2, 2-CTA backward); same results up to the order of the dq reductions.
  */

@@ -3,13 +3,12 @@
 // Three implementations of the main step exist:
 //   fused   one kernel per key tile with five MMAs (paper Section 3.2); dQ is reduced into an FP32
 //           accumulator with bulk (TMA) reduce-adds.  Fastest; dQ's summation order is not fixed.
-//           Head dimension 128 only.
 //   pair    the same step on clusters of two CTAs with tcgen05 cta_group::2 MMAs (the paper's 2-CTA
 //           backward): 3/4 of the operand traffic and half of the dQ reductions.  Head dimension 128.
 //   split   bwd_dkdv_kernel + bwd_dq_kernel: no global reductions, every output bit-reproducible,
 //           no accumulator in the workspace; recomputes S and dP once more (7 MMAs).
-// Default: fused for D = 128, split for D = 64.  FA_BWD_IMPL=split | pair (read once per process)
-// selects the others; split works for every head dimension.
+// Default: fused.  FA_BWD_IMPL=split | pair (read once per process) selects the others; pair is for
+// head dimension 128 only.
 #include "fa_bwd_fused.cuh"
 #include "fa_bwd_kernels.cuh"
 #include "fa_bwd_pair.cuh"
@@ -24,7 +23,7 @@ static bool bwd_use_fused(const Shape& s) {
     const char* e = getenv("FA_BWD_IMPL");
     return e && strcmp(e, "split") == 0;
   }();
-  return s.D == 128 && !force_split && !s.deterministic;
+  return !force_split && !s.deterministic;
 }
 
 // FA_BWD_IMPL=pair (read once): the fused step runs on CTA pairs (bwd_pair_kernel) instead of single CTAs.
@@ -56,7 +55,11 @@ static BwdWorkspace bwd_layout(const Shape& s) {
 size_t bwd_workspace_bytes(const Shape& s) { return bwd_layout(s).total; }
 
 // Shared-memory opt-in of the fused kernel (dense and packed launches share it), per device.
-static PerDeviceFlag g_attr_fused_bf16, g_attr_fused_f16;
+template <int D, bool kF16>
+static int fused_smem_once() {
+  static PerDeviceFlag done;
+  return set_smem_once(bwd_fused_kernel<D, kF16>, (int)sizeof(BwdFusedSmem<D>), done);
+}
 
 // The two split kernels: dK/dV per key tile, then dQ per query tile.
 template <int D, bool kF16, typename Preprocess>
@@ -81,7 +84,7 @@ template <int D>
 static int bwd_launch_d(const void* q, const void* k, const void* v, const void* o, const float* lse, const void* d_o,
                         void* dq, void* dk, void* dv, const Shape& s, void* workspace, cudaStream_t stream) {
   const bool fused = bwd_use_fused(s);
-  if (s.f16 && fused && bwd_use_pair()) return FA_ERR_UNSUPPORTED;  // the CTA-pair kernel is BF16 only
+  if (s.f16 && fused && D == 128 && bwd_use_pair()) return FA_ERR_UNSUPPORTED;  // the CTA-pair kernel is BF16 only
   const BwdWorkspace w = bwd_layout(s);
   float* dq_acc = fused ? static_cast<float*>(workspace) : nullptr;
   float* delta = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + w.dq_acc_bytes);
@@ -129,9 +132,10 @@ static int bwd_launch_d(const void* q, const void* k, const void* v, const void*
     return cudaGetLastError() == cudaSuccess ? FA_OK : FA_ERR_CUDA;
   };
 
-  if constexpr (D == 128) {
-    if (fused) {
-      // 2. fused main kernel, 3. accumulator -> bf16 dQ
+  if (fused) {
+    // 2. fused main kernel, 3. accumulator -> 16-bit dQ
+    bool launched = false;
+    if constexpr (D == 128) {
       if (bwd_use_pair()) {
         CUtensorMap tq64, tdo64;
         if ((st = encode_bshd_map(&tq64, q, s.B, s.Sq, s.H, D, 64, 64, bf16, 2, sw)) != FA_OK) return st;
@@ -144,24 +148,21 @@ static int bwd_launch_d(const void* q, const void* k, const void* v, const void*
         bwd_pair_kernel<<<(unsigned)n_pair_ctas, 512, sizeof(BwdPairSmem), stream>>>(tq, tq64, tk, tv, tdo, tdo64, tdk,
                                                                                       tdv, p, n_kv_pairs);
         if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
-      } else if (s.f16) {
-        if ((st = set_smem_once(bwd_fused_kernel<true>, (int)sizeof(BwdFusedSmem), g_attr_fused_f16)) != FA_OK) return st;
-        if ((st = preprocess()) != FA_OK) return st;
-        bwd_fused_kernel<true><<<(unsigned)n_kv_ctas, 512, sizeof(BwdFusedSmem), stream>>>(tq, tk, tv, tdo, tdk, tdv, p,
-                                                                                          n_kv_tiles);
-        if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
-      } else {
-        if ((st = set_smem_once(bwd_fused_kernel<false>, (int)sizeof(BwdFusedSmem), g_attr_fused_bf16)) != FA_OK) return st;
-        if ((st = preprocess()) != FA_OK) return st;
-        bwd_fused_kernel<false><<<(unsigned)n_kv_ctas, 512, sizeof(BwdFusedSmem), stream>>>(tq, tk, tv, tdo, tdk, tdv, p,
-                                                                                           n_kv_tiles);
-        if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
+        launched = true;
       }
-      auto conv = s.f16 ? bwd_convert_dq_chunked_kernel<true> : bwd_convert_dq_chunked_kernel<false>;
-      conv<<<(unsigned)conv_blocks, 256, 0, stream>>>(dq_acc, static_cast<__nv_bfloat16*>(dq), n8, s.scale, s.H, s.Sq,
-                                                 w.sq_pad);
-      return cudaGetLastError() == cudaSuccess ? FA_OK : FA_ERR_CUDA;
     }
+    if (!launched) {
+      st = s.f16 ? fused_smem_once<D, true>() : fused_smem_once<D, false>();
+      if (st != FA_OK) return st;
+      if ((st = preprocess()) != FA_OK) return st;
+      auto kernel = s.f16 ? bwd_fused_kernel<D, true> : bwd_fused_kernel<D, false>;
+      kernel<<<(unsigned)n_kv_ctas, 512, sizeof(BwdFusedSmem<D>), stream>>>(tq, tk, tv, tdo, tdk, tdv, p, n_kv_tiles);
+      if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
+    }
+    auto conv = s.f16 ? bwd_convert_dq_chunked_kernel<D, true> : bwd_convert_dq_chunked_kernel<D, false>;
+    conv<<<(unsigned)conv_blocks, 256, 0, stream>>>(dq_acc, static_cast<__nv_bfloat16*>(dq), n8, s.scale, s.H, s.Sq,
+                                                    w.sq_pad);
+    return cudaGetLastError() == cudaSuccess ? FA_OK : FA_ERR_CUDA;
   }
   // 2a. dK, dV;  2b. dQ
   if (s.f16) return bwd_split_launch<D, true>(tq, tk, tv, tdo, tdq, tdk, tdv, p, n_kv_tiles, n_q_tiles, preprocess, stream);
@@ -212,8 +213,7 @@ int bwd_varlen_launch(const void* q, const void* k, const void* v, const void* o
   const size_t n8 = (size_t)total_q * s.H * D / 8;
   const size_t conv_blocks = (n8 + 255) / 256;
   if (pre_blocks > 0x7fffffffll || n_ctas > 0x7fffffffll || conv_blocks > 0x7fffffffull) return FA_ERR_UNSUPPORTED;
-  st = s.f16 ? set_smem_once(bwd_fused_kernel<true>, (int)sizeof(BwdFusedSmem), g_attr_fused_f16)
-             : set_smem_once(bwd_fused_kernel<false>, (int)sizeof(BwdFusedSmem), g_attr_fused_bf16);
+  st = s.f16 ? fused_smem_once<D, true>() : fused_smem_once<D, false>();
   if (st != FA_OK) return st;
 
   varlen_pad_offsets_kernel<<<1, 32, 0, stream>>>(cu_q, s.B, pad_off);
@@ -237,13 +237,8 @@ int bwd_varlen_launch(const void* q, const void* k, const void* v, const void* o
   p.total_pad = tp;
   p.dk = static_cast<__nv_bfloat16*>(dk);
   p.dv = static_cast<__nv_bfloat16*>(dv);
-  if (s.f16) {
-    bwd_fused_kernel<true><<<(unsigned)n_ctas, 512, sizeof(BwdFusedSmem), stream>>>(tq, tk, tv, tdo, tdk, tdv, p,
-                                                                                   n_kv_tiles);
-  } else {
-    bwd_fused_kernel<false><<<(unsigned)n_ctas, 512, sizeof(BwdFusedSmem), stream>>>(tq, tk, tv, tdo, tdk, tdv, p,
-                                                                                    n_kv_tiles);
-  }
+  auto kernel = s.f16 ? bwd_fused_kernel<D, true> : bwd_fused_kernel<D, false>;
+  kernel<<<(unsigned)n_ctas, 512, sizeof(BwdFusedSmem<D>), stream>>>(tq, tk, tv, tdo, tdk, tdv, p, n_kv_tiles);
   if (cudaGetLastError() != cudaSuccess) return FA_ERR_CUDA;
   auto conv = s.f16 ? bwd_convert_dq_varlen_kernel<true> : bwd_convert_dq_varlen_kernel<false>;
   conv<<<(unsigned)conv_blocks, 256, 0, stream>>>(dq_acc, static_cast<__nv_bfloat16*>(dq), n8, s.scale, cu_q, pad_off,

@@ -1,15 +1,19 @@
 // Backward main kernel, single-kernel ("fused") form of the paper's Section 3.2 for head
-// dimension 128: five MMAs per (key tile, query tile) pair with P and dS resident in tensor
-// memory, dQ reduced into an FP32 global accumulator.
+// dimensions 128 and 64: five MMAs per (key tile, query tile) pair with P and dS resident in
+// tensor memory, dQ reduced into an FP32 global accumulator.
 //
 // Differences from the generic kernel in fa_bwd_kernels.cuh:
-//   * dQ^T (head dim x queries) is drained by four warps, each owning 32 head-dim rows.  A warp
-//     copies a 32-query chunk (32 x 32 floats, 4 KiB) into its private shared-memory slot with
+//   * The dQ tile is drained by four warps that work independently.  A warp copies a chunk of 32
+//     queries x 32 head dims (4 KiB of floats) into its private shared-memory slot with
 //     conflict-free stores and hands it to the TMA unit as ONE bulk reduce-add.  The accumulator
-//     layout [B][H][Sq_pad/32][4][32][32] makes that chunk contiguous in global memory, so the L2
-//     receives whole 128-byte lines (the pattern it reduces fastest) and the SM's load/store pipe
-//     is not clogged by reduction instructions.  Slots are double-buffered per warp; nothing is
-//     synchronised across warps.
+//     layout [B][H][Sq_pad/32][D/32][32][32] makes that chunk contiguous in global memory, so the
+//     L2 receives whole 128-byte lines (the pattern it reduces fastest) and the SM's load/store
+//     pipe is not clogged by reduction instructions.  Slots are double-buffered per warp.
+//     D = 128: the product is formed transposed, dQ^T = K^T dS^T (head dim on the tensor-memory
+//     lanes, over the dP^T / dS^T region), a warp owns 32 head dims of all 128 queries and a chunk
+//     is stored [query][head dim].  D = 64: dQ = dS K with the queries on the lanes, in a region
+//     of its own (tensor memory has room), a warp owns 32 queries and a chunk is stored
+//     [head dim][query].
 //   * dO_i is single-buffered (it is free again once dV += P^T dO_i has been issued), which pays
 //     for the 32 KiB of reduction slots; Delta_i travels with Q_i.
 #pragma once
@@ -18,13 +22,15 @@
 
 namespace fa {
 
+template <int D>
 struct BwdFusedSmem {
-  static constexpr int kTileBytes = 128 * 128 * 2;
+  static constexpr int kTileBytes = 128 * D * 2;
+  static constexpr int kDsBytes = 128 * 128 * 2;
   alignas(1024) uint8_t k[kTileBytes];
   alignas(1024) uint8_t v[kTileBytes];
   alignas(1024) uint8_t q[2][kTileBytes];  // Q_i stages; q[0] stages dK in the epilogue
   alignas(1024) uint8_t d_o[kTileBytes];   // dO_i (single stage); stages dV in the epilogue
-  alignas(1024) uint8_t ds[kTileBytes];    // dS^T tile, [key row][query], 128-byte swizzle
+  alignas(1024) uint8_t ds[kDsBytes];      // dS^T tile, [key row][query], 128-byte swizzle
   alignas(1024) float red_slot[4][2][32 * 32];  // [warp][buffer][query][head dim]: one 4 KiB bulk reduce each
   alignas(16) float lse2[2][128];
   alignas(16) float delta[2][128];
@@ -35,52 +41,65 @@ struct BwdFusedSmem {
   WaitCtl ctl;  // abort flag and launch epoch, read by every bounded wait
 };
 
-// dQ accumulator element (b, h, q, d) in the chunked layout the bulk reductions use.
+// dQ accumulator element (b, h, q, d) in the chunked layout the bulk reductions use: chunks of 32
+// queries x 32 head dims; inside a chunk [query][head dim] for D = 128, [head dim][query] for D = 64.
+template <int D>
 __host__ __device__ inline size_t dq_acc_chunked_index(int b, int h, int q, int d, int H, int Sq_pad) {
-  return ((((size_t)b * H + h) * (Sq_pad / 32) + q / 32) * 4 + d / 32) * 1024 + (size_t)(q % 32) * 32 + d % 32;
+  const size_t chunk = (((size_t)b * H + h) * (Sq_pad / 32) + q / 32) * (D / 32) + d / 32;
+  return chunk * 1024 + (D == 128 ? (size_t)(q % 32) * 32 + d % 32 : (size_t)(d % 32) * 32 + q % 32);
 }
 
-template <bool kF16>
+template <int D, bool kF16>
 __global__ void __launch_bounds__(256)
 bwd_convert_dq_chunked_kernel(const float* __restrict__ dq_acc, __nv_bfloat16* __restrict__ dq, size_t n8, float scale,
                               int H, int Sq, int Sq_pad) {
-  // idx runs over groups of 8 elements of dq [B, Sq, H, 128]
+  // idx runs over groups of 8 elements of dq [B, Sq, H, D]
   const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= n8) return;
-  const int sub = (int)(idx % 16);
-  const int h = (int)((idx / 16) % H);
-  const int q = (int)((idx / ((size_t)16 * H)) % Sq);
-  const int bb = (int)(idx / ((size_t)16 * H * Sq));
-  const float4* src = reinterpret_cast<const float4*>(dq_acc + dq_acc_chunked_index(bb, h, q, sub * 8, H, Sq_pad));
-  const float4 a = src[0], b = src[1];
+  constexpr int kSubs = D / 8;
+  const int sub = (int)(idx % kSubs);
+  const int h = (int)((idx / kSubs) % H);
+  const int q = (int)((idx / ((size_t)kSubs * H)) % Sq);
+  const int bb = (int)(idx / ((size_t)kSubs * H * Sq));
+  float x[8];
+  if (D == 128) {
+    const float4* src = reinterpret_cast<const float4*>(dq_acc + dq_acc_chunked_index<D>(bb, h, q, sub * 8, H, Sq_pad));
+    const float4 a = src[0], b = src[1];
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+  } else {
+    const float* src = dq_acc + dq_acc_chunked_index<D>(bb, h, q, sub * 8, H, Sq_pad);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) x[e] = src[e * 32];  // consecutive head dims are 32 floats apart
+  }
   uint4 w;
-  w.x = pack2<kF16>(a.x * scale, a.y * scale);
-  w.y = pack2<kF16>(a.z * scale, a.w * scale);
-  w.z = pack2<kF16>(b.x * scale, b.y * scale);
-  w.w = pack2<kF16>(b.z * scale, b.w * scale);
+  w.x = pack2<kF16>(x[0] * scale, x[1] * scale);
+  w.y = pack2<kF16>(x[2] * scale, x[3] * scale);
+  w.z = pack2<kF16>(x[4] * scale, x[5] * scale);
+  w.w = pack2<kF16>(x[6] * scale, x[7] * scale);
   reinterpret_cast<uint4*>(dq)[idx] = w;
 }
 
-template <bool kF16>  // inputs and outputs FP16 instead of BF16
+template <int D, bool kF16>  // kF16: inputs and outputs FP16 instead of BF16
 __global__ void __launch_bounds__(512, 1)
 bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
                  const __grid_constant__ CUtensorMap tm_dk, const __grid_constant__ CUtensorMap tm_dv,
                  const BwdParams p, const int n_kv_tiles) {
-  constexpr int D = 128;
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  using Smem = BwdFusedSmem;
+  using Smem = BwdFusedSmem<D>;
   Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
   if ((smem_u32(smem_raw) & 1023u) != 0) {
     if (threadIdx.x == 0) record_device_status(5, __LINE__, p.epoch);
     return;
   }
-  constexpr int kRegions = 2;
+  constexpr int kRegions = D / 64;
   constexpr int kRegionBytes = 128 * 128;
   constexpr uint32_t kIdescSS = make_idesc(128, 128, false, false, kF16);
   constexpr uint32_t kIdescAcc = make_idesc(128, D, false, true, kF16);
-  constexpr uint32_t kIdescDqT = make_idesc(128, 128, true, true, kF16);
-  constexpr uint32_t kColR0 = 0, kColR1 = 128, kColDv = 256, kColDk = 384;
+  // D = 128: dQ^T = K^T dS^T (128 head dims x 128 queries); D = 64: dQ = dS K (128 queries x 64 head dims)
+  constexpr uint32_t kIdescDq = make_idesc(128, D == 128 ? 128 : 64, true, true, kF16);
+  constexpr uint32_t kColR0 = 0, kColR1 = 128, kColDv = 256, kColDk = 256 + D;
+  constexpr uint32_t kColDq = D == 128 ? kColR1 : 256 + 2 * D;  // D = 64: a region of its own
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* abort_flag = &sm.ctl.abort_flag;
@@ -252,11 +271,11 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       if (ok) {
 #pragma unroll
         for (int which = 0; which < 2; ++which) {
-          const uint32_t acc_addr = tmem + (which == 0 ? kColDv : kColDk) + lane_base + wg * 64;
+          const uint32_t acc_addr = tmem + (which == 0 ? kColDv : kColDk) + lane_base + wg * (D / 2);
           uint8_t* stage_buf = which == 0 ? sm.d_o : sm.q[0];
           const float mul = which == 0 ? 1.0f : p.scale;
 #pragma unroll
-          for (int cc = 0; cc < 2; ++cc) {
+          for (int cc = 0; cc < D / 64; ++cc) {
             uint32_t v[32];
             if (n_iter > 0) {
               tmem_ld32(acc_addr + cc * 32, v);
@@ -265,7 +284,8 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll
               for (int e = 0; e < 32; ++e) v[e] = 0u;
             }
-            uint8_t* row_ptr = stage_buf + wg * kRegionBytes + r * 128;
+            // this warpgroup's half of the head dims: a 64-column region of its own (D = 128) or half a region (D = 64)
+            uint8_t* row_ptr = stage_buf + (D == 128 ? wg * kRegionBytes : 0) + r * 128;
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
               uint4 w4;
@@ -273,12 +293,12 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
               w4.y = pack2<kF16>(__uint_as_float(v[8 * ch + 2]) * mul, __uint_as_float(v[8 * ch + 3]) * mul);
               w4.z = pack2<kF16>(__uint_as_float(v[8 * ch + 4]) * mul, __uint_as_float(v[8 * ch + 5]) * mul);
               w4.w = pack2<kF16>(__uint_as_float(v[8 * ch + 6]) * mul, __uint_as_float(v[8 * ch + 7]) * mul);
-              const int chunk = cc * 4 + ch;
+              const int chunk = D == 128 ? cc * 4 + ch : wg * 4 + ch;  // 16-byte chunk inside the 128-byte row
               if (kv_tail) {
                 // the rows after this sequence's last key belong to the next sequence: no 128-row TMA store,
                 // every valid row is written on its own
                 __nv_bfloat16* out = (which == 0 ? p.dv : p.dk) +
-                                     ((size_t)(k_row0 + min(key, Sk - 1)) * p.Hkv + hk) * D + wg * 64 + chunk * 8;
+                                     ((size_t)(k_row0 + min(key, Sk - 1)) * p.Hkv + hk) * D + (D == 128 ? wg * 64 : 0) + chunk * 8;
                 if (key < Sk) *reinterpret_cast<uint4*>(out) = w4;
               } else {
                 *reinterpret_cast<uint4*>(row_ptr + ((chunk ^ (r & 7)) << 4)) = w4;
@@ -306,7 +326,8 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     // ============================================================ dQ reduction warps (independent of one another)
     reg_dealloc<80>();
     const int w = warp & 3;
-    const uint32_t addr = tmem + kColR1 + ((uint32_t)(w * 32) << 16);  // this thread: head-dim row 32w + lane
+    // this thread: head-dim row 32w + lane of dQ^T (D = 128), query 32w + lane of dQ (D = 64)
+    const uint32_t addr = tmem + kColDq + ((uint32_t)(w * 32) << 16);
     bool ok = true;
     for (int it = 0; it < n_iter && ok; ++it) {
       const int h = hk * group + it / iters_per_head;
@@ -314,17 +335,17 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       ok = __all_sync(0xffffffffu, mbar_wait(&sm.dq_full, it & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
-      // global chunk (32 queries x this warp's 32 head dims) = 4 KiB contiguous
-      float* dst = p.dq_acc + (((acc_row0 + (size_t)h * acc_head_stride) / 32 + (size_t)i * 4) * 4 + w) * 1024;
-      // two chunks (both slots) at a time, so that the region is handed back after two rounds of stores, not three
+      // first 32-query chunk of the tile in the accumulator (chunks of 4 KiB, D / 32 per 32 queries)
+      float* tile_dst = p.dq_acc + ((acc_row0 + (size_t)h * acc_head_stride) / 32 + (size_t)i * 4) * (D / 32) * 1024;
+      // two chunks (both slots) per round
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
+      for (int half = 0; half < D / 64; ++half) {
         uint32_t v[2][32];
         tmem_ld32(addr + half * 64, v[0]);
         tmem_ld32(addr + half * 64 + 32, v[1]);
         tmem_wait_ld();
-        if (half == 1) {
-          // everything is in registers: the next dP^T may overwrite the region
+        if (half == D / 64 - 1) {
+          // everything is in registers: the region may be overwritten
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(&sm.dq_drained);
@@ -343,8 +364,10 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         if (lane == 0) {
 #pragma unroll
           for (int s2 = 0; s2 < 2; ++s2) {
-            asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;" ::"l"(
-                             dst + (size_t)(half * 2 + s2) * 4096),
+            // D = 128: queries [32 (2 half + s2), +32) x this warp's head dims; D = 64: this warp's queries x head dims [32 s2, +32)
+            float* dst = D == 128 ? tile_dst + ((size_t)(half * 2 + s2) * 4 + w) * 1024
+                                  : tile_dst + ((size_t)w * 2 + s2) * 1024;
+            asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;" ::"l"(dst),
                          "r"(smem_u32(sm.red_slot[w][s2])), "r"(4096)
                          : "memory");
           }
@@ -396,7 +419,8 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         for (int it = 0; it < n_iter; ++it) {
           const int stage = it & 1;
           if (!(ok = wait_bar(&sm.do_full, it & 1))) break;
-          if (it > 0 && !(ok = wait_bar(&sm.dq_drained, (it - 1) & 1))) break;
+          // D = 128: dQ^T of the previous tile sits in this region until the drain warps hold it in registers
+          if (D == 128 && it > 0 && !(ok = wait_bar(&sm.dq_drained, (it - 1) & 1))) break;
           tc_fence_after();
           ss_kmajor(kColR1, v_lo, do_lo, &sm.dp_full);  // dP^T(it)
           if (!(ok = wait_bar(&sm.p_ready, it & 1))) break;
@@ -413,11 +437,19 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
           ts_acc(kColDk, kColR1, q_mn_lo0 + stage * kStageStep, it > 0 ? 1u : 0u);  // dK += dS^T Q
           if (!(ok = wait_bar(&sm.ds_ready, it & 1))) break;
           tc_fence_after();
+          // D = 64: dQ has a region of its own, free again once the drain warps hold the previous tile
+          if (D == 64 && it > 0 && !(ok = wait_bar(&sm.dq_drained, (it - 1) & 1))) break;
+          if (D == 64) tc_fence_after();
           if (elect_one()) {
 #pragma unroll
-            for (int kk = 0; kk < 8; ++kk)  // dQ^T = K^T dS^T: rows = head dim, columns = queries
-              mma_ss_lohi(tmem + kColR1, k_mn_lo + ((kk * 2048) >> 4), ds_mn_lo + ((kk * 2048) >> 4), kDescHiSw128,
-                          kIdescDqT, kk > 0);
+            for (int kk = 0; kk < 8; ++kk) {
+              if (D == 128)  // dQ^T = K^T dS^T: rows = head dim, columns = queries
+                mma_ss_lohi(tmem + kColDq, k_mn_lo + ((kk * 2048) >> 4), ds_mn_lo + ((kk * 2048) >> 4), kDescHiSw128,
+                            kIdescDq, kk > 0);
+              else  // dQ = dS K: rows = queries (A = dS^T read transposed), columns = head dim
+                mma_ss_lohi(tmem + kColDq, ds_mn_lo + ((kk * 2048) >> 4), k_mn_lo + ((kk * 2048) >> 4), kDescHiSw128,
+                            kIdescDq, kk > 0);
+            }
             mma_commit(&sm.dq_full);
             mma_commit(&sm.q_empty[stage]);
           }

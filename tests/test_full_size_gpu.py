@@ -138,3 +138,27 @@ def test_config5_backward(S, causal):
         for name, got, want in zip(("dq", "dk", "dv"), (dq, dk, dv), ref):
             err = np.abs(to_f64(got[b, :, h, :]) - want).max()
             assert err <= GRAD_RTOL * np.abs(want).max(), (name, b, h, err, np.abs(want).max())
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_backward_head_dim_64_full_size(causal):
+    """The D = 64 shape of the head-dim sweep (32 heads, 8192 tokens, batch 2) through the backward pass:
+    whole heads of dQ, dK and dV against the oracle."""
+    import torch
+
+    from paper_2603_05451_b200 import binding
+
+    B, H, S, D = 2, 32, 8192, 64
+    t = _tensors(6000, B, H, H, S, D, with_do=True)
+    scale = D ** -0.5
+    q, k, v, d_o = (to_dev(t[n][0]) for n in ("q", "k", "v", "do"))
+    o, lse = binding.fa_fwd(q, k, v, scale, causal)
+    dq, dk, dv = binding.fa_bwd(q, k, v, o, lse, d_o, scale, causal)
+    torch.cuda.synchronize()
+    assert binding.fa_last_device_status() == 0
+    for b, h in _whole_heads(B, H, 2):
+        qh, kh, vh, doh = (_f64(t[n][0][b, :, h, :]) for n in ("q", "k", "v", "do"))
+        ref = attn_bwd_head(qh, kh, vh, doh, scale, causal)
+        for name, got, want in zip(("dq", "dk", "dv"), (dq, dk, dv), ref):
+            err = np.abs(to_f64(got[b, :, h, :]) - want).max()
+            assert err <= GRAD_RTOL * np.abs(want).max(), (name, b, h, err, np.abs(want).max())
