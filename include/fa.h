@@ -196,6 +196,13 @@ int fa_last_device_status(void* stream);
 int fa_exp2_emulated(const float* x, float* y, size_t n, void* stream);
 
 /*
+ * Test hook, host only (no GPU needed): exercises the per-device bookkeeping behind the
+ * "once per device ordinal" set-up named in the conventions above.  Returns FA_OK if flags of
+ * different ordinals are independent and out-of-range ordinals are ignored.
+ */
+int fa_selftest_per_device_flags(void);
+
+/*
  * Test hook for the bounded waits: launches one warp that waits on a barrier nobody arrives on.  The
  * wait gives up after its limit (about half a second), the kernel ends normally, and the next
  * fa_last_device_status() returns FA_ERR_DEVICE_TIMEOUT once; the context stays usable.

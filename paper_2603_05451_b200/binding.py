@@ -65,6 +65,8 @@ def lib():
         l.fa_last_device_status.restype = i
         l.fa_exp2_emulated.argtypes = [vp, vp, sz, vp]
         l.fa_exp2_emulated.restype = i
+        l.fa_selftest_per_device_flags.argtypes = []
+        l.fa_selftest_per_device_flags.restype = i
         l.fa_selftest_unsatisfied_wait.argtypes = [vp]
         l.fa_selftest_unsatisfied_wait.restype = i
         _lib = l

@@ -303,6 +303,23 @@ int fa_exp2_emulated(const float* x, float* y, size_t n, void* stream) {
   return cudaGetLastError() == cudaSuccess ? FA_OK : FA_ERR_CUDA;
 }
 
+int fa_selftest_per_device_flags(void) {
+  // Host-only check of the per-device bookkeeping: flags of different device ordinals are independent,
+  // out-of-range ordinals read as "not set" and are ignored when set.
+  static PerDeviceFlag f;
+  if (f.test(0) || f.test(1) || f.test(-1) || f.test(kMaxDevices)) return FA_ERR_INVALID_ARGUMENT;
+  f.set(1, 2);
+  if (f.test(0) || !f.test(1) || f.get(1) != 2 || f.get(0) != 0) return FA_ERR_INVALID_ARGUMENT;
+  f.set(kMaxDevices);
+  f.set(-1);
+  if (f.test(kMaxDevices) || f.test(-1) || f.get(kMaxDevices) != 0) return FA_ERR_INVALID_ARGUMENT;
+  f.set(0);
+  if (!f.test(0) || !f.test(1) || f.test(2)) return FA_ERR_INVALID_ARGUMENT;
+  f.set(0, 0);
+  f.set(1, 0);
+  return FA_OK;
+}
+
 int fa_selftest_unsatisfied_wait(void* stream) {
   int st = check_device();
   if (st != FA_OK) return st;

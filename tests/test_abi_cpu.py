@@ -74,3 +74,9 @@ def test_no_gpu_means_an_error_not_a_fallback(binding):
         pytest.skip("a GPU is present")
     st = binding.fa_fwd_raw(0x1000, 0x2000, 0x3000, 0x4000, 0x5000, 1, 2, 2, 128, 128, 128, 0.1, 0)
     assert st in (2, 3)
+
+
+def test_per_device_bookkeeping_is_independent_per_ordinal(binding):
+    """Function attributes and the architecture check are cached per device ordinal; the host-only
+    self-test walks two ordinals and the out-of-range cases."""
+    assert binding.lib().fa_selftest_per_device_flags() == 0
