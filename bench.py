@@ -127,10 +127,10 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def workload_text(with_bwd, masks, seqlens, long_member):
+def workload_text(with_bwd, masks, seqlens, long_member, D=HEAD_DIM):
     mask_txt = {"both": "non-causal and causal", "causal": "causal", "noncausal": "non-causal"}[masks]
     long_txt = f", plus the causal forward at seqlen {LONG_SEQLEN} (batch 1)" if long_member else ""
-    return (f"{'fwd+bwd' if with_bwd else 'fwd'} {mask_txt} D=128 H=16, 16384 total tokens, seqlen sweep "
+    return (f"{'fwd+bwd' if with_bwd else 'fwd'} {mask_txt} D={D} H={HEADS * HEAD_DIM // D}, 16384 total tokens, seqlen sweep "
             f"{','.join(map(str, seqlens))} (batch = 16384/seqlen){long_txt}")
 
 
@@ -254,6 +254,8 @@ def main():
     ap.add_argument("--masks", default="both", choices=["both", "causal", "noncausal"])
     ap.add_argument("--seqlens", default=",".join(str(s) for s in SEQLENS))
     ap.add_argument("--no-long", action="store_true", help="leave out the causal forward at seqlen 32768")
+    ap.add_argument("--head-dim", type=int, default=HEAD_DIM, choices=[64, 128],
+                    help="head dimension (hidden size 2048: 16 heads of 128, the headline; or 32 heads of 64, for profiles)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--table", action="store_true",
                     help="print forward / backward TFLOPs/s over head dim 64/128, seqlen 1k-32k, causal and not, and exit")
@@ -285,7 +287,8 @@ def main():
 
     seqlens = [int(s) for s in args.seqlens.split(",")]
     masks = {"both": (False, True), "causal": (True,), "noncausal": (False,)}[args.masks]
-    H, D = HEADS, HEAD_DIM
+    D = args.head_dim
+    H = HEADS * HEAD_DIM // D
     scale = D ** -0.5
     with_bwd = args.which == "fwdbwd"
     # The step's members: (seqlen, batch, causal, backward too?)
@@ -512,7 +515,7 @@ def main():
         "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {
-            "workload": workload_text(with_bwd, args.masks, seqlens, members[-1][0] == LONG_SEQLEN),
+            "workload": workload_text(with_bwd, args.masks, seqlens, members[-1][0] == LONG_SEQLEN, D),
             "inputs": "i.i.d. N(0,1) bf16, seeded; Q+K+V+O = 256 MiB per launch, larger than the 126 MB L2 (no flush)",
             "multi_gpu": "replicas only: every rank runs the same workload, no collective on the data path",
         },
