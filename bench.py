@@ -34,9 +34,10 @@ METRIC = "attention fwd/bwd TFLOPs/s (BF16, D=128, causal & non) and % of B200 B
 # each from the one ncu capture named beside it (a 16384-token member of the sweep; compulsory traffic
 # depends on the token count only, K/V re-reads are served by L2).
 NCU_TRAFFIC = {
-    "fwd": {"bytes": 235.4e6 + 59.7e6,
-            "capture": "profiles/ncu_fwd_pipe_kernel_S4096_B4_H16_D128.txt (one launch, B=4 S=4096 non-causal)"},
-    "bwd": {"bytes": 404.9e6 + 223.4e6,
+    "fwd": {"bytes": 260.57e6 + 59.53e6,
+            "capture": "profiles/ncu_fwd_pipe_kernel_S4096_B4_H16_D128.txt (one launch, B=4 S=4096 non-causal; "
+                       "the causal launch of the same shape: 202.1e6 + 51.2e6)"},
+    "bwd": {"bytes": 405.28e6 + 226.70e6,
             "capture": "profiles/ncu_bwd_fused_kernel_S4096_B4_H16_D128.txt (one launch, B=4 S=4096 non-causal)"},
 }
 ROOFLINE_KERNEL = {
