@@ -1,6 +1,7 @@
 // Forward-pass launch code: builds the tensor maps and launches the kernel.
 #include "fa_common.cuh"
 #include "fa_fwd_pipe.cuh"
+#include "fa_fwd_tile.cuh"
 
 namespace fa {
 
@@ -18,6 +19,9 @@ static int make_maps(CUtensorMap* tq, CUtensorMap* tk, CUtensorMap* tv, CUtensor
 
 // Default share of exponentials computed on the FMA pipe, per head dimension (of every 8).
 constexpr int kDefaultEmuPer8D64 = 0, kDefaultEmuPer8D128 = 0;
+// Longest key sequence that goes to the one-tile-per-CTA kernel: the measured crossover with the pipelined
+// kernel at 16384 tokens per launch, per head dimension and mask.
+constexpr int kTileMaxSkD128 = 512, kTileMaxSkCausalD128 = 1024, kTileMaxSkD64 = 1024, kTileMaxSkCausalD64 = 2048;
 
 static FwdParams make_params(void* o, float* lse, const Shape& s) {
   FwdParams p;
@@ -68,12 +72,48 @@ static int launch_pipe(const CUtensorMap& tq, const CUtensorMap& tk, const CUten
   return cudaGetLastError() == cudaSuccess ? FA_OK : FA_ERR_CUDA;
 }
 
+// One launch of the one-tile-per-CTA kernel (two CTAs per SM).
+template <int D, int kEmuPer8, bool kF16>
+static int launch_tile(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& to,
+                       const FwdParams& p, const Shape& s, cudaStream_t stream) {
+  static PerDeviceFlag attr_set, carveout_set;
+  constexpr int smem = fwd_tile_smem_bytes<D>();
+  auto kernel = fwd_tile_kernel<D, kEmuPer8, kF16>;
+  const int n_mblocks = (s.Sq + 127) / 128;
+  const long long n_ctas = (long long)s.B * s.H * n_mblocks;
+  if (n_ctas > 0x7fffffffll) return FA_ERR_UNSUPPORTED;
+  int st = set_smem_once(kernel, smem, attr_set);
+  if (st != FA_OK) return st;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FA_ERR_CUDA;
+  if (!carveout_set.test(dev)) {  // two CTAs of ~100 KiB each must fit: ask for the largest shared-memory split
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) !=
+        cudaSuccess)
+      return FA_ERR_CUDA;
+    carveout_set.set(dev);
+  }
+  kernel<<<(unsigned)n_ctas, 256, smem, stream>>>(tq, tk, tv, to, p, n_mblocks);
+  return cudaGetLastError() == cudaSuccess ? FA_OK : FA_ERR_CUDA;
+}
+
+// Which kernel a dense call gets.  The one-tile kernel hides the per-CTA set-up and epilogue behind a second
+// resident CTA but reads K and V twice as often; it wins while a tile has few key blocks.  FA_FWD_TILE (read
+// once per process): 0 = never, 1 = always, unset = by sequence length.
+static bool use_tile_kernel(const Shape& s) {
+  static const int forced = env_int("FA_FWD_TILE", -1);
+  if (forced >= 0) return forced != 0;
+  const int max_sk = s.D == 64 ? (s.causal ? kTileMaxSkCausalD64 : kTileMaxSkD64)
+                               : (s.causal ? kTileMaxSkCausalD128 : kTileMaxSkD128);
+  return s.Sk <= max_sk;
+}
+
 template <int D, int kEmuPer8, bool kF16 = false>
 static int launch_dense(const void* q, const void* k, const void* v, void* o, float* lse, const Shape& s,
                         cudaStream_t stream) {
   CUtensorMap tq, tk, tv, to;
   int st = make_maps(&tq, &tk, &tv, &to, q, k, v, o, s);
   if (st != FA_OK) return st;
+  if (use_tile_kernel(s)) return launch_tile<D, kEmuPer8, kF16>(tq, tk, tv, to, make_params(o, lse, s), s, stream);
   return launch_pipe<D, D, kEmuPer8, kF16>(tq, tk, tv, to, make_params(o, lse, s), s, stream);
 }
 

@@ -145,11 +145,28 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   const int n_max = max(n_blk[0], n_blk[1]);
   const int n_blk_mine = (warp >> 2) == 1 ? n_blk[1] : n_blk[0];  // softmax warps: blocks of their tile
 
+  auto load_q = [&](int t) {
+    if (n_blk[t] > 0) {
+      mbar_expect_tx(&sm.q_full[t], Smem::kQkTileBytes);
+      for (int r = 0; r < kQkRegions; ++r)
+        tma_load_4d(sm.q[t] + r * kRegionBytes, &tm_q, &sm.q_full[t], r * 64, tile.h, q_row0 + tile.m0 + t * 128, tma_b);
+    }
+  };
+  auto load_k = [&](int j, int slot) {
+    mbar_expect_tx(&sm.k_full[slot], Smem::kQkTileBytes);
+    for (int r = 0; r < kQkRegions; ++r)
+      tma_load_4d(sm.k[slot] + r * kRegionBytes, &tm_k, &sm.k_full[slot], r * 64, tile.hk, k_row0 + j * 128, tma_b);
+  };
+  auto load_v = [&](int j, int slot) {
+    mbar_expect_tx(&sm.v_full[slot], Smem::kVTileBytes);
+    for (int r = 0; r < kRegions; ++r)
+      tma_load_4d(sm.v[slot] + r * kRegionBytes, &tm_v, &sm.v_full[slot], r * 64, tile.hk, k_row0 + j * 128, tma_b);
+  };
+
   if (tid == 0) {
     sm.ctl.abort_flag = 0;
     sm.ctl.launch_epoch = (int)p.epoch;
     for (int t = 0; t < 2; ++t) {
-      mbar_init(&sm.q_full[t], 1);
       mbar_init(&sm.s_full[t], 1);
       mbar_init(&sm.p_full[t], 8);  // 4 softmax warps + 4 correction warps
       mbar_init(&sm.p_last[t], 4);
@@ -158,14 +175,8 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       for (int w = 0; w < 4; ++w) mbar_init(&sm.stat_full[t][w], 1);
       for (int w = 0; w < 4; ++w) mbar_init(&sm.fin_full[t][w], 1);
     }
-    for (int s = 0; s < kKStages; ++s) {
-      mbar_init(&sm.k_full[s], 1);
-      mbar_init(&sm.k_empty[s], 1);
-    }
-    for (int s = 0; s < kVStages; ++s) {
-      mbar_init(&sm.v_full[s], 1);
-      mbar_init(&sm.v_empty[s], 1);
-    }
+    for (int s = 0; s < kKStages; ++s) mbar_init(&sm.k_empty[s], 1);
+    for (int s = 0; s < kVStages; ++s) mbar_init(&sm.v_empty[s], 1);
     mbar_init(&sm.s_free, 4);
     fence_barrier_init();
   }
@@ -174,9 +185,20 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     tmem_relinquish();
   }
   if (warp == 13 && lane == 0) {
-    tma_prefetch_desc(&tm_q);
-    tma_prefetch_desc(&tm_k);
-    tma_prefetch_desc(&tm_v);
+    // The producer arms the barriers its loads complete on by itself and sends the first loads off at
+    // once, while tensor memory is still being allocated: what the first products need first.
+    for (int t = 0; t < 2; ++t) mbar_init(&sm.q_full[t], 1);
+    for (int s = 0; s < kKStages; ++s) mbar_init(&sm.k_full[s], 1);
+    for (int s = 0; s < kVStages; ++s) mbar_init(&sm.v_full[s], 1);
+    fence_barrier_init();
+    if (n_max > 0) {
+      load_q(0);
+      load_k(0, 0);
+      load_q(1);
+      load_v(0, 0);
+      for (int j = 1; j < kKStages && j < n_max; ++j) load_k(j, j);
+      for (int j = 1; j < kVStages && j < n_max; ++j) load_v(j, j);
+    }
     tma_prefetch_desc(&tm_o);
   }
   tc_fence_before();
@@ -493,31 +515,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // ============================================================ TMA producer
     reg_dealloc<48>();
     if (n_max > 0 && lane == 0) {
-      auto load_q = [&](int t) {
-        if (n_blk[t] > 0) {
-          mbar_expect_tx(&sm.q_full[t], Smem::kQkTileBytes);
-          for (int r = 0; r < kQkRegions; ++r)
-            tma_load_4d(sm.q[t] + r * kRegionBytes, &tm_q, &sm.q_full[t], r * 64, tile.h, q_row0 + tile.m0 + t * 128,
-                        tma_b);
-        }
-      };
-      auto load_k = [&](int j, int slot) {
-        mbar_expect_tx(&sm.k_full[slot], Smem::kQkTileBytes);
-        for (int r = 0; r < kQkRegions; ++r)
-          tma_load_4d(sm.k[slot] + r * kRegionBytes, &tm_k, &sm.k_full[slot], r * 64, tile.hk, k_row0 + j * 128, tma_b);
-      };
-      auto load_v = [&](int j, int slot) {
-        mbar_expect_tx(&sm.v_full[slot], Smem::kVTileBytes);
-        for (int r = 0; r < kRegions; ++r)
-          tma_load_4d(sm.v[slot] + r * kRegionBytes, &tm_v, &sm.v_full[slot], r * 64, tile.hk, k_row0 + j * 128, tma_b);
-      };
-      // Fill both rings at once, what the first products need first.
-      load_q(0);
-      load_k(0, 0);
-      load_q(1);
-      load_v(0, 0);
-      for (int j = 1; j < kKStages && j < n_max; ++j) load_k(j, j);
-      for (int j = 1; j < kVStages && j < n_max; ++j) load_v(j, j);
+      // (the rings were filled before the CTA-wide barrier, see above)
       // Steady state, in the order in which the MMA warp releases stages: K_0's after the first S
       // products, then for every block j K_{j+1}'s (S_1(j+1) issued) and V_j's (both P V_j issued).
       int next_k = kKStages, next_v = kVStages;

@@ -8,6 +8,8 @@ tolerances.
 
   FA_EMU_PER8 = 1, 2, 3    that many of every 8 exponentials on the FMA pipe (Section 3.1.3)
   FA_FWD_SECTION_MB = 0, 1  all heads in one launch section / sections of one key-value head (Section 3.3)
+  FA_FWD_TILE = 0, 1        the pipelined kernel (256 rows per CTA) / the one-tile kernel (128 rows per CTA,
+                            two CTAs per SM) for every dense shape, whatever its length
 """
 
 import json
@@ -31,7 +33,8 @@ from tests.test_fwd_gpu import _fwd_case
 cases = [(1, 1, 1, 128, 128, 64, False, 1.0), (2, 2, 2, 333, 333, 128, True, 1.0), (1, 3, 3, 300, 77, 128, True, 1.0),
          (1, 2, 2, 1024, 1024, 128, False, 1.0), (1, 2, 2, 1024, 1024, 64, True, 1.0), (2, 8, 2, 640, 640, 128, True, 1.0),
          (1, 4, 1, 200, 1100, 64, True, 1.0), (1, 2, 2, 1, 700, 128, False, 1.0), (1, 2, 2, 1536, 1536, 128, True, 3.0),
-         (1, 2, 2, 1536, 1536, 64, False, 3.0), (4, 4, 4, 2048, 2048, 128, True, 1.0)]
+         (1, 2, 2, 1536, 1536, 64, False, 3.0), (4, 4, 4, 2048, 2048, 128, True, 1.0), (3, 2, 1, 129, 257, 128, False, 1.0),
+         (2, 3, 3, 255, 255, 64, True, 1.0), (1, 2, 2, 2, 1, 128, True, 1.0), (8, 16, 4, 512, 512, 128, True, 1.0)]
 out = []
 for idx, c in enumerate(cases):
     eo, el = _fwd_case(*c[:7], seed=8100 + idx, mult=c[7], v_mult=1.0)
@@ -41,10 +44,13 @@ print("RESULT " + json.dumps(out))
 
 
 @pytest.mark.parametrize("name,value", [("FA_EMU_PER8", "1"), ("FA_EMU_PER8", "2"), ("FA_EMU_PER8", "3"),
-                                        ("FA_FWD_SECTION_MB", "0"), ("FA_FWD_SECTION_MB", "1")])
+                                        ("FA_FWD_SECTION_MB", "0"), ("FA_FWD_SECTION_MB", "1"),
+                                        ("FA_FWD_TILE", "0"), ("FA_FWD_TILE", "1"),
+                                        ("FA_FWD_TILE+FA_EMU_PER8", "1+2")])
 def test_forward_variants_match_the_oracle(name, value):
     env = dict(os.environ)
-    env[name] = value
+    for n, v in zip(name.split("+"), value.split("+")):
+        env[n] = v
     res = subprocess.run([sys.executable, "-c", CHILD % {"root": ROOT}], env=env, capture_output=True, text=True,
                          timeout=900, cwd=ROOT)
     assert res.returncode == 0, res.stderr[-2000:]
