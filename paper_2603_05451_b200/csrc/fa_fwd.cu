@@ -17,11 +17,11 @@ static int make_maps(CUtensorMap* tq, CUtensorMap* tk, CUtensorMap* tv, CUtensor
   return FA_OK;
 }
 
-// Default share of exponentials computed on the FMA pipe, per head dimension (of every 8).
-constexpr int kDefaultEmuPer8D64 = 0, kDefaultEmuPer8D128 = 0;
 // Longest key sequence that goes to the one-tile-per-CTA kernel: the measured crossover with the pipelined
 // kernel at 16384 tokens per launch, per head dimension and mask.
-constexpr int kTileMaxSkD128 = 512, kTileMaxSkCausalD128 = 1024, kTileMaxSkD64 = 1024, kTileMaxSkCausalD64 = 2048;
+// At D = 64 that kernel keeps P in tensor-memory columns of its own; without a mask it is the faster one at
+// every length measured (to 32768), with the causal mask up to 4096 keys.
+constexpr int kTileMaxSkD128 = 512, kTileMaxSkCausalD128 = 1024, kTileMaxSkD64 = 1 << 30, kTileMaxSkCausalD64 = 4096;
 
 static FwdParams make_params(void* o, float* lse, const Shape& s) {
   FwdParams p;
@@ -131,12 +131,14 @@ int fwd_hd192_launch(const void* q, const void* k, const void* v, void* o, float
   return launch_pipe<192, 128, 0, false>(tq, tk, tv, to, make_params(o, lse, s), s, stream);
 }
 
-// How many of every 8 exponentials use the software 2^x (Section 3.1.3).  The default is chosen per
-// head dimension; FA_EMU_PER8 = 0..3 (read once per process) overrides it for both.
-static int emu_per8(int D) {
+// How many of every 8 exponentials use the software 2^x (Section 3.1.3).  The default is the measured best per
+// kernel, head dimension and mask: 1 of 8 where the exponential unit is the limit and nothing else is in the
+// way (D = 64 in the one-tile kernel, no mask: +2 ... +6 %), none elsewhere.  FA_EMU_PER8 = 0..3 (read once per
+// process) overrides it for every call.
+static int emu_per8(const Shape& s) {
   static const int forced = env_int("FA_EMU_PER8", -1);
   if (forced >= 0) return forced > 3 ? 3 : forced;
-  return D == 64 ? kDefaultEmuPer8D64 : kDefaultEmuPer8D128;
+  return (s.D == 64 && !s.causal && use_tile_kernel(s)) ? 1 : 0;
 }
 
 int fwd_launch(const void* q, const void* k, const void* v, void* o, float* lse, const Shape& s, cudaStream_t stream) {
@@ -144,7 +146,7 @@ int fwd_launch(const void* q, const void* k, const void* v, void* o, float* lse,
     return s.D == 64 ? launch_dense<64, 0, true>(q, k, v, o, lse, s, stream)
                      : launch_dense<128, 0, true>(q, k, v, o, lse, s, stream);
   }
-  const int emu = emu_per8(s.D);
+  const int emu = emu_per8(s);
   if (s.D == 64) {
     switch (emu) {
       case 1: return launch_dense<64, 1>(q, k, v, o, lse, s, stream);

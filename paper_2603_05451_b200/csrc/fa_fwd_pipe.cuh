@@ -66,9 +66,11 @@ __device__ __forceinline__ int fwd_num_blocks(int Sq, int Sk, int causal, int m_
 
 template <int D, int kEmuPer8, bool kF16>
 __device__ __forceinline__ void softmax_exp_chunk(const uint32_t (&s)[32], uint32_t (&out)[16], float c, float neg_mc,
-                                                  float2& sum2) {
+                                                  float2& sum2, float x_top, bool& top_emulated) {
   // 32 scores -> 16 packed pairs of 16-bit probabilities (bf16, or fp16 when kF16).  Of every 8 elements, kEmuPer8 use the
-  // software 2^x on the FMA pipe (Section 3.1.3, partial emulation), the rest MUFU.EX2.
+  // software 2^x on the FMA pipe (Section 3.1.3, partial emulation), the rest MUFU.EX2.  `top_emulated` is raised when an
+  // emulated element has the exponent `x_top` of the block's largest score: the row-sum compensation of the caller has to
+  // round the very value that was stored for that element.
   const float2 c2 = make_float2(c, c), m2 = make_float2(neg_mc, neg_mc);
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
@@ -77,9 +79,19 @@ __device__ __forceinline__ void softmax_exp_chunk(const uint32_t (&s)[32], uint3
     const bool emu0 = ((2 * i) & 7) < kEmuPer8, emu1 = ((2 * i + 1) & 7) < kEmuPer8;
     e.x = emu0 ? exp2_emulated(x.x) : ex2_approx(x.x);
     e.y = emu1 ? exp2_emulated(x.y) : ex2_approx(x.y);
+    if (emu0) top_emulated |= x.x == x_top;
+    if (emu1) top_emulated |= x.y == x_top;
     sum2 = __fadd2_rn(sum2, e);
     out[i] = pack2<kF16>(e.x, e.y);
   }
+}
+// What rounding to 16 bits added to the block's largest probability (exponent x_top), computed the way the element
+// itself was (see softmax_exp_chunk).
+template <int kEmuPer8, bool kF16>
+__device__ __forceinline__ float top_rounding_excess(float x_top, bool top_emulated) {
+  float p_top = ex2_approx(x_top);
+  if (kEmuPer8 > 0 && top_emulated) p_top = exp2_emulated(x_top);
+  return unpack2<kF16>(pack2<kF16>(p_top, 0.0f)).x - p_top;
 }
 
 // D: value / output head dimension; kF16: inputs and output are FP16 instead of BF16
@@ -293,15 +305,13 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       if (lane == 0) mbar_arrive(&sm.stat_full[t][w]);
 
       const float neg_mc = (m_run == -INFINITY) ? 0.0f : -m_run * c;
-      {
-        const float p_top = ex2_approx(fmaf(m_blk, c, neg_mc));  // the block's largest probability, as computed below
-        l_fix += unpack2<kF16>(pack2<kF16>(p_top, 0.0f)).x - p_top;
-      }
+      const float x_top = fmaf(m_blk, c, neg_mc);  // exponent of the block's largest probability, as formed below
+      bool top_emulated = false;
       float2 sum2 = make_float2(0.0f, 0.0f);
 #pragma unroll
       for (int q4 = 0; q4 < 4; ++q4) {
         uint32_t pk[16];
-        softmax_exp_chunk<D, kEmuPer8, kF16>(s[q4], pk, c, neg_mc, sum2);
+        softmax_exp_chunk<D, kEmuPer8, kF16>(s[q4], pk, c, neg_mc, sum2, x_top, top_emulated);
         tmem_st16(p_addr + q4 * 16, pk);
         if (q4 == 2) {
           // staged store: three quarters of P are enough to start O += P V
@@ -312,6 +322,7 @@ fwd_pipe_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
       }
       l_run += sum2.x + sum2.y;
+      l_fix += top_rounding_excess<kEmuPer8, kF16>(x_top, top_emulated);
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();

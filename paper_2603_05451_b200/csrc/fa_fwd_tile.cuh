@@ -15,10 +15,13 @@
 //   warp 4     issues every tcgen05.mma:  S = Q K_j^T,  O += P V_j  (P read from tensor memory)
 //   warp 5     TMA producer: Q once, then K_j and V_j through mbarrier rings
 //   warps 6-7  idle (they only donate registers)
-// Tensor memory (256 columns): S [0,128), overwritten in place by the 16-bit P [0,64) once a thread holds
-// its row of scores in registers (the paper's layout); O [128,128+D).  S(j+1) is issued behind O += P(j) V_j
+// Tensor memory (256 columns), D = 128: S [0,128), overwritten in place by the 16-bit P [0,64) once a thread
+// holds its row of scores in registers (the paper's layout); O [128,256).  S(j+1) is issued behind O += P(j) V_j
 // on the same in-order pipe, so it cannot overtake the read of P(j), and its completion implies that of
 // that product: the softmax warps need no further barrier before they touch O.
+// D = 64: O takes 64 columns, which leaves P a place of its own: S [0,128), P [128,192), O [192,256).  S(j+1) is
+// then issued as soon as S(j) has been read into registers (s_free), i.e. under the softmax of block j, and the
+// softmax warps wait for O += P(j-1) V_{j-1} (o_full) before they rescale O or overwrite P.
 #pragma once
 
 #include "fa_fwd_pipe.cuh"
@@ -35,9 +38,10 @@ struct FwdTileSmem {
   alignas(8) uint64_t q_full;
   uint64_t k_full[kStages], k_empty[kStages];
   uint64_t v_full[kStages], v_empty[kStages];
-  uint64_t s_full;    // MMA -> softmax: S(j) is in tensor memory (and O += P(j-1) V_{j-1} has finished)
+  uint64_t s_full;    // MMA -> softmax: S(j) is in tensor memory (D = 128: and O += P(j-1) V_{j-1} has finished)
+  uint64_t s_free;    // softmax -> MMA (D = 64): S(j) has been read into registers
   uint64_t p_full;    // softmax -> MMA: P(j) stored, O rescaled if that was needed
-  uint64_t o_full;    // MMA -> softmax: the last O += P V has finished
+  uint64_t o_full;    // MMA -> softmax: O += P(j) V_j has finished
   uint64_t o_staged;  // softmax warps -> storing thread: the O tile is in shared memory
   uint32_t tmem_base;
   WaitCtl ctl;  // abort flag and launch epoch, read by every bounded wait
@@ -60,6 +64,8 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   constexpr int kRegionBytes = 128 * 128;
   constexpr uint32_t kIdescS = make_idesc(128, 128, false, false, kF16);
   constexpr uint32_t kIdescO = make_idesc(128, D, false, true, kF16);
+  constexpr bool kSeparateP = D == 64;  // P in columns of its own (see the layout above)
+  constexpr uint32_t kColP = kSeparateP ? 128u : 0u, kColO = kSeparateP ? 192u : 128u;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* abort_flag = &sm.ctl.abort_flag;
@@ -97,6 +103,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     sm.ctl.abort_flag = 0;
     sm.ctl.launch_epoch = (int)p.epoch;
     mbar_init(&sm.s_full, 1);
+    mbar_init(&sm.s_free, 4);
     mbar_init(&sm.p_full, 4);
     mbar_init(&sm.o_full, 1);
     mbar_init(&sm.o_staged, 4);
@@ -139,7 +146,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int r_in_tile = w * 32 + lane;
     const int row = m0 + r_in_tile;
     const uint32_t s_addr = tmem + ((uint32_t)(w * 32) << 16);
-    const uint32_t o_addr = s_addr + 128u;
+    const uint32_t p_addr = s_addr + kColP, o_addr = s_addr + kColO;
     const float c = p.scale_log2;
     const int shift = Sk - Sq;
     const int row_limit = p.causal ? min(Sk - 1, row + shift) : Sk - 1;  // last visible key
@@ -166,7 +173,14 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
       for (int q4 = 0; q4 < 4; ++q4) {
-        if (q4 == 2) tmem_wait_ld();
+        if (q4 == 2) {
+          tmem_wait_ld();
+          if (kSeparateP) {  // the score buffer may be overwritten by the next block's product
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.s_free);
+          }
+        }
         if (masked) {
 #pragma unroll
           for (int i = 0; i < 32; ++i)
@@ -185,12 +199,18 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       // Conditional rescale (Eq. 6): only when the maximum grew by more than tau in the base-2
       // domain; the decision is taken for the whole warp (Section 3.1.4, last sentence).
       const bool need = (m_new - m_run) * c > p.tau;
+      if (kSeparateP && j > 0) {
+        // O += P(j-1) V_{j-1} has finished: O may be rescaled and P overwritten
+        ok = __all_sync(0xffffffffu, mbar_wait(&sm.o_full, (j - 1) & 1, abort_flag, __LINE__));
+        if (!ok) break;
+        tc_fence_after();
+      }
       if (__any_sync(0xffffffffu, need)) {
         const float f = (m_run == -INFINITY) ? 0.0f : ex2_approx((m_run - m_new) * c);
         l_run *= f;
         l_fix *= f;
         m_run = m_new;
-        if (j > 0) {  // O holds the sum over blocks 0..j-1 (s_full(j) came after that product)
+        if (j > 0) {  // O holds the sum over blocks 0..j-1
 #pragma unroll
           for (int cc = 0; cc < D / 32; ++cc) {
             uint32_t r[32];
@@ -203,18 +223,17 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
       }
       const float neg_mc = (m_run == -INFINITY) ? 0.0f : -m_run * c;
-      {
-        const float p_top = ex2_approx(fmaf(m_blk, c, neg_mc));  // the block's largest probability, as computed below
-        l_fix += unpack2<kF16>(pack2<kF16>(p_top, 0.0f)).x - p_top;
-      }
+      const float x_top = fmaf(m_blk, c, neg_mc);  // exponent of the block's largest probability, as formed below
+      bool top_emulated = false;
       float2 sum2 = make_float2(0.0f, 0.0f);
 #pragma unroll
       for (int q4 = 0; q4 < 4; ++q4) {
         uint32_t pk[16];
-        softmax_exp_chunk<D, kEmuPer8, kF16>(s[q4], pk, c, neg_mc, sum2);
-        tmem_st16(s_addr + q4 * 16, pk);  // P over the first half of this row's scores, all of which are in registers
+        softmax_exp_chunk<D, kEmuPer8, kF16>(s[q4], pk, c, neg_mc, sum2, x_top, top_emulated);
+        tmem_st16(p_addr + q4 * 16, pk);  // (D = 128: over the first half of this row's scores, all in registers)
       }
       l_run += sum2.x + sum2.y;
+      l_fix += top_rounding_excess<kEmuPer8, kF16>(x_top, top_emulated);
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();
@@ -225,7 +244,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       const float inv_l = l_run > 0.0f ? 1.0f / (l_run + l_fix) : 0.0f;
       if (row < Sq) p.lse[((size_t)b * p.H + h) * Sq + row] = l_run > 0.0f ? (m_run * c + log2f(l_run)) * kLn2 : -INFINITY;
       if (n > 0) {
-        ok = __all_sync(0xffffffffu, mbar_wait(&sm.o_full, 0, abort_flag, __LINE__));
+        ok = __all_sync(0xffffffffu, mbar_wait(&sm.o_full, (n - 1) & 1, abort_flag, __LINE__));
         tc_fence_after();
       }
       if (ok) {
@@ -295,6 +314,11 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       do {
         if (!(wait_bar(&sm.q_full, 0) && do_s(0))) break;
         for (int j = 0; j < n; ++j) {
+          if (kSeparateP && j + 1 < n) {  // S(j+1) under the softmax of block j
+            if (!wait_bar(&sm.s_free, j & 1)) break;
+            tc_fence_after();
+            if (!do_s(j + 1)) break;
+          }
           const int slot = j % kStages;
           if (!wait_bar(&sm.v_full[slot], (uint32_t)((j / kStages) & 1))) break;
           if (!wait_bar(&sm.p_full, j & 1)) break;
@@ -303,13 +327,13 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
           if (elect_one()) {  // O += P V_j
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk)
-              mma_ts_lohi(tmem + 128u, tmem + kk * 8, b_lo + ((kk * 2048) >> 4), kDescHiSw128, kIdescO,
+              mma_ts_lohi(tmem + kColO, tmem + kColP + kk * 8, b_lo + ((kk * 2048) >> 4), kDescHiSw128, kIdescO,
                           kk > 0 ? 1u : (j > 0 ? 1u : 0u));
             mma_commit(&sm.v_empty[slot]);
-            if (j == n - 1) mma_commit(&sm.o_full);
+            mma_commit(&sm.o_full);
           }
           __syncwarp();
-          if (j + 1 < n && !do_s(j + 1)) break;
+          if (!kSeparateP && j + 1 < n && !do_s(j + 1)) break;
         }
       } while (false);
     }

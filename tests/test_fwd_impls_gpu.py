@@ -69,3 +69,14 @@ def test_fa_log_names_the_wait_that_gave_up():
                          timeout=300, cwd=ROOT)
     assert res.returncode == 0, res.stderr[-2000:]
     assert "device-side wait expired (code 5, site" in res.stderr
+
+
+@pytest.mark.parametrize("emu", ["1", "3"])
+def test_emulated_exponentials_hold_the_tolerance_on_the_wide_score_configuration(emu):
+    """Config 4 at full size (Q and K scaled by 3: most rows put their weight on one key, so the rounding of
+    the largest probability shows in O) with part of the exponentials on the FMA pipe: the row-sum
+    compensation has to round the value that was actually stored, whichever unit produced it."""
+    res = subprocess.run([sys.executable, "-m", "pytest", "tests/test_full_size_gpu.py", "-x", "-q", "-m", "gpu", "-k",
+                          "config4"], env=dict(os.environ, FA_EMU_PER8=emu), capture_output=True, text=True,
+                         timeout=1800, cwd=ROOT)
+    assert res.returncode == 0, res.stdout[-3000:]
