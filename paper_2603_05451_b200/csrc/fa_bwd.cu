@@ -113,6 +113,11 @@ static int bwd_launch_d(const void* q, const void* k, const void* v, const void*
   p.epoch = next_launch_epoch();
   const int n_kv_tiles = (s.Sk + 127) / 128;
   const int n_q_tiles = (s.Sq + 127) / 128;
+  // Causal mask: launch order in sections of a few heads, longest key tiles of a section first (see the fused
+  // kernel).  Measured at 16384 tokens, 16 heads of 128: sections of 8 heads +1 ... +5 % up to 8192 keys, of 4 heads
+  // +3 % at 16384; whole-launch longest-first order loses the L2 sharing of Q and dO between the tiles of a head
+  // (-15 % at 1024 keys).
+  if (s.causal) p.heads_per_section = n_kv_tiles > 64 ? 4 : 8;
   const long long n_kv_ctas = (long long)n_kv_tiles * s.Hkv * s.B;
   const long long n_q_ctas = (long long)n_q_tiles * s.H * s.B;
   // Every size check comes before the first launch: on an error nothing has been launched.

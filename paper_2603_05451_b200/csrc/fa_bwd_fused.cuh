@@ -104,9 +104,27 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* abort_flag = &sm.ctl.abort_flag;
 
-  const int n_tile = blockIdx.x % n_kv_tiles;
-  const int hk = (blockIdx.x / n_kv_tiles) % p.Hkv;
-  const int b = blockIdx.x / (n_kv_tiles * p.Hkv);
+  // Launch order.  Without a mask every key tile costs the same and the tiles of one (batch, head) follow each
+  // other, so that the CTAs in flight stream the same Q and dO.  With the causal mask the first key tile of a
+  // sequence meets every query tile and the last one a single one; a head's long tiles that start late would
+  // leave the other SMs idle at the end.  The launch code then asks for sections of a few heads: inside a section
+  // the key-tile index is the slow coordinate, so the section's longest tiles start first and its shortest fill the
+  // tail (longest-processing-time-first, Section 3.3), while the tiles of a head still run close enough together
+  // to share their Q and dO reads in L2.
+  int n_tile, hk, b;
+  if (p.heads_per_section > 0) {
+    const int heads = p.Hkv * p.B, per_section = p.heads_per_section * n_kv_tiles;
+    const int sec = blockIdx.x / per_section, r = blockIdx.x % per_section;
+    const int g = min(p.heads_per_section, heads - sec * p.heads_per_section);  // the last section may be smaller
+    n_tile = r / g;
+    const int hb = sec * p.heads_per_section + r % g;
+    hk = hb % p.Hkv;
+    b = hb / p.Hkv;
+  } else {
+    n_tile = blockIdx.x % n_kv_tiles;
+    hk = (blockIdx.x / n_kv_tiles) % p.Hkv;
+    b = blockIdx.x / (n_kv_tiles * p.Hkv);
+  }
   const int j0 = n_tile * 128;
   const int group = p.H / p.Hkv;
   // Dense batch: sequence b of length Sq / Sk at batch coordinate b.  Packed batch: this sequence's

@@ -33,6 +33,9 @@ struct BwdParams {
   float scale, scale_log2;
   int causal;
   unsigned epoch;  // identifies this launch in the device status word (bounded waits)
+  // Fused kernel, causal dense batches: launch order in sections of this many (batch, key/value head) pairs,
+  // inside a section the key tiles from the longest down (0: no sections, the key tiles of a head in a row).
+  int heads_per_section = 0;
   // Variable-length batches (fused kernel only; null / 0 otherwise): sequence b owns query tokens
   // [cu_q[b], cu_q[b+1]) and key tokens [cu_k[b], cu_k[b+1]) of the packed tensors; in the workspace
   // arrays (accumulator, lse2, delta: [H, total_pad, ...]) its rows start at pad_off[b], a multiple
