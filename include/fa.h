@@ -50,7 +50,12 @@ enum {
 
 /*
  * Forward pass (paper Section 2.1, first display; kernel design Section 3.1).
- * Reads q, k, v; overwrites o (bfloat16) and lse (float32).  One kernel launch on `stream`.
+ * Reads q, k, v; overwrites o (bfloat16) and lse (float32).  One kernel launch on `stream`: short key
+ * sequences (and D = 64 at most lengths) get a kernel with one 128-row tile per thread block and two
+ * blocks per SM, the others one with two tiles per block that take turns on the tensor cores; both
+ * compute the same thing (FA_FWD_TILE=0 or 1 in the environment, read at the first call, forces the
+ * second or the first kernel for every call; FA_EMU_PER8=0..3 likewise fixes how many of every eight
+ * exponentials are computed by the polynomial of Section 3.1.3 instead of the hardware unit).
  * Forward results are bit-reproducible from run to run.
  * Arithmetic: scores and all accumulation in FP32; the probabilities enter the second product
  * rounded to 16 bits, scaled by 2^-(running maximum) with the maximum refreshed only when it grew
