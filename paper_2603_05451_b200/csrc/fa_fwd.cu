@@ -207,6 +207,16 @@ int fwd_varlen_launch(const void* q, const void* k, const void* v, void* o, floa
   CUtensorMap tq, tk, tv, to;
   int st = make_maps(&tq, &tk, &tv, &to, q, k, v, o, packed);
   if (st != FA_OK) return st;
+  // Choice of the kernel: half the longest query length stands for the typical key length (the call has no bound
+  // on the key lengths, and in a batch of mixed lengths most sequences are well below the longest), so batches of
+  // short sequences go to the one-tile kernel like short dense calls.  Measured at 16 heads of 128: 32 lengths of
+  // 64...2048 causal +12 %, 64 of 64...1024 +2...6 % / +20 % (causal), 128 of 32...512 +10 % / +25 %.
+  Shape longest = s;
+  longest.Sk = (s.Sq + 1) / 2;
+  if (use_tile_kernel(longest)) {
+    if (s.D == 64) return launch_tile<64, 0, false>(tq, tk, tv, to, p, s, stream);
+    return launch_tile<128, 0, false>(tq, tk, tv, to, p, s, stream);
+  }
   if (s.D == 64) return launch_pipe<64, 64, 0, false>(tq, tk, tv, to, p, s, stream);
   return launch_pipe<128, 128, 0, false>(tq, tk, tv, to, p, s, stream);
 }

@@ -73,8 +73,10 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
   // Work decode: batches outermost, then sections of heads whose K and V fit in L2 together, then
   // 128-row tiles from the LAST one down (longest causal tiles first, Section 3.3), the heads of the
   // section fastest so the heads sharing K/V run together.
-  const int Sq = p.Sq, Sk = p.Sk;
+  int Sq = p.Sq, Sk = p.Sk;   // for a variable-length batch: this sequence's lengths (set below)
   int b, h, hk, m0;
+  int q_row0 = 0, k_row0 = 0;  // token-axis origin of this sequence in the tensor maps
+  float* lse_rows;             // LSE of (this sequence, this head), indexed by the row inside the sequence
   {
     const int idx = blockIdx.x;
     const int hs = p.heads_per_section > 0 ? p.heads_per_section : p.H;
@@ -85,18 +87,32 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     h = (r / per_section) * hs + r2 % hs;
     m0 = (n_mblocks - 1 - r2 / hs) * 128;
     hk = h / (p.H / p.Hkv);
+    if (p.cu_q != nullptr) {
+      // Packed sequences (Section 3.3, variable sequence length): virtual batch index -> sequence in
+      // longest-first order; tiles past the end of a short sequence leave at once.
+      const int seq = p.order != nullptr ? p.order[b] : b;
+      q_row0 = p.cu_q[seq];
+      k_row0 = p.cu_k[seq];
+      Sq = p.cu_q[seq + 1] - q_row0;
+      Sk = p.cu_k[seq + 1] - k_row0;
+      if (m0 >= Sq) return;
+      b = 0;  // batch coordinate of the packed tensors
+      lse_rows = p.lse + (size_t)h * p.total_q + q_row0;
+    } else {
+      lse_rows = p.lse + ((size_t)b * p.H + h) * Sq;
+    }
   }
   const int n = fwd_num_blocks(Sq, Sk, p.causal, m0);
 
   auto load_k = [&](int j, int slot) {
     mbar_expect_tx(&sm.k_full[slot], Smem::kTileBytes);
     for (int r = 0; r < kRegions; ++r)
-      tma_load_4d(sm.k[slot] + r * kRegionBytes, &tm_k, &sm.k_full[slot], r * 64, hk, j * 128, b);
+      tma_load_4d(sm.k[slot] + r * kRegionBytes, &tm_k, &sm.k_full[slot], r * 64, hk, k_row0 + j * 128, b);
   };
   auto load_v = [&](int j, int slot) {
     mbar_expect_tx(&sm.v_full[slot], Smem::kTileBytes);
     for (int r = 0; r < kRegions; ++r)
-      tma_load_4d(sm.v[slot] + r * kRegionBytes, &tm_v, &sm.v_full[slot], r * 64, hk, j * 128, b);
+      tma_load_4d(sm.v[slot] + r * kRegionBytes, &tm_v, &sm.v_full[slot], r * 64, hk, k_row0 + j * 128, b);
   };
 
   if (tid == 0) {
@@ -128,7 +144,7 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     fence_barrier_init();
     if (n > 0) {
       mbar_expect_tx(&sm.q_full, Smem::kTileBytes);
-      for (int r = 0; r < kRegions; ++r) tma_load_4d(sm.q + r * kRegionBytes, &tm_q, &sm.q_full, r * 64, h, m0, b);
+      for (int r = 0; r < kRegions; ++r) tma_load_4d(sm.q + r * kRegionBytes, &tm_q, &sm.q_full, r * 64, h, q_row0 + m0, b);
       for (int j = 0; j < kStages && j < n; ++j) load_k(j, j);
       for (int j = 0; j < kStages && j < n; ++j) load_v(j, j);
     }
@@ -242,13 +258,17 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     if (ok && m0 < Sq) {
       const float inv_l = l_run > 0.0f ? 1.0f / (l_run + l_fix) : 0.0f;
-      if (row < Sq) p.lse[((size_t)b * p.H + h) * Sq + row] = l_run > 0.0f ? (m_run * c + log2f(l_run)) * kLn2 : -INFINITY;
+      if (row < Sq) lse_rows[row] = l_run > 0.0f ? (m_run * c + log2f(l_run)) * kLn2 : -INFINITY;
       if (n > 0) {
         ok = __all_sync(0xffffffffu, mbar_wait(&sm.o_full, (n - 1) & 1, abort_flag, __LINE__));
         tc_fence_after();
       }
       if (ok) {
         uint8_t* stage = sm.q;  // no product reads Q any more
+        // In a packed batch the rows after a sequence's last one belong to the next sequence, so a tile
+        // that overhangs the end cannot leave through a 128-row TMA store: its rows are written one by one.
+        const bool row_by_row = p.cu_q != nullptr && m0 + 128 > Sq;
+        __nv_bfloat16* o_row = p.o + ((size_t)(q_row0 + min(row, Sq - 1)) * p.H + h) * D;
 #pragma unroll
         for (int cc = 0; cc < D / 32; ++cc) {
           uint32_t r[32];
@@ -269,18 +289,25 @@ fwd_tile_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             v4.z = pack2<kF16>(__uint_as_float(r[8 * i + 4]) * inv_l, __uint_as_float(r[8 * i + 5]) * inv_l);
             v4.w = pack2<kF16>(__uint_as_float(r[8 * i + 6]) * inv_l, __uint_as_float(r[8 * i + 7]) * inv_l);
             const int chunk = (cc & 1) * 4 + i;
-            *reinterpret_cast<uint4*>(region + ((chunk ^ (r_in_tile & 7)) << 4)) = v4;
+            if (row_by_row) {
+              if (row < Sq) reinterpret_cast<uint4*>(o_row + cc * 32)[i] = v4;
+            } else {
+              *reinterpret_cast<uint4*>(region + ((chunk ^ (r_in_tile & 7)) << 4)) = v4;
+            }
           }
         }
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.o_staged);
-        if (w == 0) {
-          ok = __all_sync(0xffffffffu, mbar_wait(&sm.o_staged, 0, abort_flag, __LINE__));
-          if (ok && lane == 0) {
-            for (int r = 0; r < kRegions; ++r) tma_store_4d(&tm_o, stage + r * kRegionBytes, r * 64, h, m0, b);
-            tma_commit_group();
-            tma_wait_group_read<0>();
+        if (!row_by_row) {  // (warp-uniform)
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sm.o_staged);
+          if (w == 0) {
+            ok = __all_sync(0xffffffffu, mbar_wait(&sm.o_staged, 0, abort_flag, __LINE__));
+            if (ok && lane == 0) {
+              for (int r = 0; r < kRegions; ++r)
+                tma_store_4d(&tm_o, stage + r * kRegionBytes, r * 64, h, q_row0 + m0, b);
+              tma_commit_group();
+              tma_wait_group_read<0>();
+            }
           }
         }
       }

@@ -80,3 +80,12 @@ def test_emulated_exponentials_hold_the_tolerance_on_the_wide_score_configuratio
                           "config4"], env=dict(os.environ, FA_EMU_PER8=emu), capture_output=True, text=True,
                          timeout=1800, cwd=ROOT)
     assert res.returncode == 0, res.stdout[-3000:]
+
+
+@pytest.mark.parametrize("tile", ["0", "1"])
+def test_packed_batches_through_either_forward_kernel(tile):
+    """The packed-batch tests (per-sequence oracle parity, ragged ends, grouped heads, longest-first order) with
+    every call forced through the pipelined kernel (0) or the one-tile kernel (1)."""
+    res = subprocess.run([sys.executable, "-m", "pytest", "tests/test_fwd_varlen_gpu.py", "-x", "-q", "-m", "gpu"],
+                         env=dict(os.environ, FA_FWD_TILE=tile), capture_output=True, text=True, timeout=1800, cwd=ROOT)
+    assert res.returncode == 0, res.stdout[-3000:]
