@@ -41,7 +41,7 @@ NCU_TRAFFIC = {
             "capture": "profiles/ncu_bwd_fused_kernel_S4096_B4_H16_D128.txt (one launch, B=4 S=4096 non-causal)"},
 }
 ROOFLINE_KERNEL = {
-    "fwd": "fwd_pipe_kernel (timed as fa_fwd: one launch)",
+    "fwd": "fwd_pipe_kernel (timed as fa_fwd: one launch; the shortest members run fwd_tile_kernel, see fa.h)",
     "bwd": "bwd_fused_kernel (timed as fa_bwd: preprocess + main + dQ conversion; the main kernel is 0.96 of it)",
 }
 
