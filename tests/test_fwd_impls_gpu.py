@@ -89,3 +89,13 @@ def test_packed_batches_through_either_forward_kernel(tile):
     res = subprocess.run([sys.executable, "-m", "pytest", "tests/test_fwd_varlen_gpu.py", "-x", "-q", "-m", "gpu"],
                          env=dict(os.environ, FA_FWD_TILE=tile), capture_output=True, text=True, timeout=1800, cwd=ROOT)
     assert res.returncode == 0, res.stdout[-3000:]
+
+
+@pytest.mark.parametrize("tile", ["0", "1"])
+def test_random_shapes_through_either_forward_kernel(tile):
+    """The seeded random problem shapes (odd head counts, unequal lengths around the tile size) with every dense
+    forward call forced through one kernel: by default most of them are short enough for the one-tile kernel."""
+    res = subprocess.run([sys.executable, "-m", "pytest", "tests/test_random_shapes_gpu.py", "-x", "-q", "-m", "gpu", "-k",
+                          "forward"], env=dict(os.environ, FA_FWD_TILE=tile), capture_output=True, text=True,
+                         timeout=1800, cwd=ROOT)
+    assert res.returncode == 0, res.stdout[-3000:]
