@@ -107,3 +107,30 @@ def test_backward_deterministic(D):
         g = got.float().cpu().numpy().astype(np.float64)
         assert got.dtype == torch.float16 and np.isfinite(g).all(), name
         assert np.abs(g - want).max() <= GRAD_RTOL * max(np.abs(want).max(), floor), name
+
+
+@pytest.mark.parametrize("D,H,S,B,causal", [(128, 16, 4096, 4, True), (64, 32, 8192, 2, False)])
+def test_benchmark_sized_launch_whole_heads(D, H, S, B, causal):
+    """FP16 at a benchmark-sized launch (16384 tokens, hidden size 2048): whole heads of O, LSE, dQ, dK, dV."""
+    import torch
+
+    from oracle.attention import attn_bwd_head, attn_fwd_head
+    from paper_2603_05451_b200 import binding
+
+    shape = (B, S, H, D)
+    q, k, v, d_o = (_half(6400 + D, n, shape) for n in ("q", "k", "v", "do"))
+    scale = D ** -0.5
+    qd, kd, vd, dod = (_dev(x[0]) for x in (q, k, v, d_o))
+    o, lse = binding.fa_fwd(qd, kd, vd, scale, causal)
+    dq, dk, dv = binding.fa_bwd(qd, kd, vd, o, lse, dod, scale, causal)
+    torch.cuda.synchronize()
+    assert binding.fa_last_device_status() == 0 and o.dtype == torch.float16 and dq.dtype == torch.float16
+    f64 = lambda x: x.float().cpu().numpy().astype(np.float64)
+    for b, h in ((0, 0), (B - 1, H - 1)):
+        qh, kh, vh, doh = (x[1][b, :, h, :] for x in (q, k, v, d_o))
+        o_ref, l_ref = attn_fwd_head(qh, kh, vh, scale, causal)
+        assert max_abs_err(f64(o[b, :, h, :]), o_ref) <= O_TOL
+        assert max_abs_err(f64(lse[b, h, :]), l_ref) <= LSE_TOL
+        for name, got, want in zip(("dq", "dk", "dv"), (dq, dk, dv), attn_bwd_head(qh, kh, vh, doh, scale, causal)):
+            err = np.abs(f64(got[b, :, h, :]) - want).max()
+            assert err <= GRAD_RTOL * np.abs(want).max(), (name, err)
