@@ -207,6 +207,24 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
       tmem_ld32(s_addr + 32, s[1]);
       tmem_wait_ld();
       const bool masked = p.causal && (j0 + 127 > i * 128 + shift);
+      // Tiles on the diagonal and the last key tile of a packed sequence: masked scores become -inf here, so that
+      // the loop below carries no per-element test for all the other tiles.
+      if (masked) {
+        const int first_visible = key - q0 - shift;  // columns below it are queries that do not see this key
+#pragma unroll
+        for (int h2 = 0; h2 < 2; ++h2) {
+#pragma unroll
+          for (int col = 0; col < 32; ++col)
+            if (h2 * 32 + col < first_visible) s[h2][col] = 0xff800000u;
+        }
+      }
+      if (kv_tail && key >= Sk) {
+#pragma unroll
+        for (int h2 = 0; h2 < 2; ++h2) {
+#pragma unroll
+          for (int col = 0; col < 32; ++col) s[h2][col] = 0xff800000u;
+        }
+      }
       float pr[2][32];
       const float4* lse4 = reinterpret_cast<const float4*>(&sm.lse2[stage][wg * 64]);
 #pragma unroll
@@ -223,10 +241,7 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int col = g * 4 + e;
-            float x = xs[e];
-            if (masked && key > q0 + h2 * 32 + col + shift) x = -INFINITY;
-            if (kv_tail && key >= Sk) x = -INFINITY;
-            pr[h2][col] = ex2_approx(x);
+            pr[h2][col] = ex2_approx(xs[e]);
           }
         }
         uint32_t pk[16];

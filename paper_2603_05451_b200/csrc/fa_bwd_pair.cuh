@@ -165,6 +165,15 @@ bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       tmem_ld32(s_addr + 32, s[1]);
       tmem_wait_ld();
       const bool masked = p.causal && (j0 + 127 > i * 128 + shift);
+      if (masked) {  // only tiles on the diagonal pay for the test
+        const int first_visible = key - q0 - shift;  // columns below it are queries that do not see this key
+#pragma unroll
+        for (int h2 = 0; h2 < 2; ++h2) {
+#pragma unroll
+          for (int col = 0; col < 32; ++col)
+            if (h2 * 32 + col < first_visible) s[h2][col] = 0xff800000u;  // -inf
+        }
+      }
       float pr[2][32];
       const float4* lse4 = reinterpret_cast<const float4*>(&sm.lse2[stage][wg * 64]);
 #pragma unroll
@@ -176,9 +185,7 @@ bwd_pair_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int col = g * 4 + e;
-            float x = fmaf(__uint_as_float(s[h2][col]), c, -ls[e]);
-            if (masked && key > q0 + h2 * 32 + col + shift) x = -INFINITY;
-            pr[h2][col] = ex2_approx(x);
+            pr[h2][col] = ex2_approx(fmaf(__uint_as_float(s[h2][col]), c, -ls[e]));
           }
         }
         uint32_t pk[16];

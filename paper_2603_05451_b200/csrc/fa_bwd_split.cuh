@@ -124,6 +124,15 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
       tmem_ld32(s_addr + 32, s[1]);
       tmem_wait_ld();
       const bool masked = p.causal && (j0 + 127 > i * 128 + shift);  // key `key` is visible to query q iff key <= q + shift
+      if (masked) {  // only tiles on the diagonal pay for the test
+        const int first_visible = key - q0 - shift;  // columns below it are queries that do not see this key
+#pragma unroll
+        for (int h2 = 0; h2 < 2; ++h2) {
+#pragma unroll
+          for (int col = 0; col < 32; ++col)
+            if (h2 * 32 + col < first_visible) s[h2][col] = 0xff800000u;  // -inf
+        }
+      }
       float pr[2][32];
       const float4* lse4 = reinterpret_cast<const float4*>(&sm.lse2[stage][wg * 64]);
 #pragma unroll
@@ -135,9 +144,7 @@ bwd_dkdv_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const int col = g * 4 + e;
-            float x = fmaf(__uint_as_float(s[h2][col]), c, -ls[e]);
-            if (masked && key > q0 + h2 * 32 + col + shift) x = -INFINITY;
-            pr[h2][col] = ex2_approx(x);
+            pr[h2][col] = ex2_approx(fmaf(__uint_as_float(s[h2][col]), c, -ls[e]));
           }
         }
         uint32_t pk[16];
@@ -442,15 +449,19 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.s_free);
       const bool masked = p.causal && (j * 128 + 127 > q0 + shift);  // key visible to `row` iff key <= row + shift
+      if (masked) {  // only tiles on the diagonal pay for the test
+        const int last_visible = row + shift - key0;  // columns above it are keys this query does not see
+#pragma unroll
+        for (int h2 = 0; h2 < 2; ++h2)
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            if (h2 * 32 + e > last_visible) s[h2][e] = 0xff800000u;  // -inf
+      }
       float pr[2][32];
 #pragma unroll
       for (int h2 = 0; h2 < 2; ++h2)
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          float x = fmaf(__uint_as_float(s[h2][e]), c, -my_lse2);
-          if (masked && key0 + h2 * 32 + e > row + shift) x = -INFINITY;
-          pr[h2][e] = ex2_approx(x);
-        }
+        for (int e = 0; e < 32; ++e) pr[h2][e] = ex2_approx(fmaf(__uint_as_float(s[h2][e]), c, -my_lse2));
       ok = __all_sync(0xffffffffu, mbar_wait(&sm.dp_full[j & 1], (j >> 1) & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
