@@ -37,7 +37,7 @@ NCU_TRAFFIC = {
     "fwd": {"bytes": 260.57e6 + 59.53e6,
             "capture": "profiles/ncu_fwd_pipe_kernel_S4096_B4_H16_D128.txt (one launch, B=4 S=4096 non-causal; "
                        "the causal launch of the same shape: 202.1e6 + 51.2e6)"},
-    "bwd": {"bytes": 405.28e6 + 226.70e6,
+    "bwd": {"bytes": 405.33e6 + 223.53e6,
             "capture": "profiles/ncu_bwd_fused_kernel_S4096_B4_H16_D128.txt (one launch, B=4 S=4096 non-causal)"},
 }
 ROOFLINE_KERNEL = {
